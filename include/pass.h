@@ -1,0 +1,206 @@
+/*
+ * pass.h - C boundary of the B200 (sm_100a) PaSS decoder-step library.
+ *
+ * PaSS = Parallel Speculative Sampling (Monea, Joulin, Grave; arXiv 2311.13581).
+ * One model call scores the tokens drafted by the previous call and, through k
+ * look-ahead embeddings appended to the input, drafts the next k tokens
+ * (Algorithm 1; section "Look-ahead embeddings"); the speculative-sampling rule
+ * of Algorithm 1 / Algorithm 2 then accepts a prefix of the drafts, resamples or
+ * adds one token, and the KV cache is cut back to what was kept (section
+ * "Baselines": the cache is updated after every call according to the number of
+ * drafted and accepted tokens).
+ *
+ * Naming: the paper writes q for the target law and p for the draft law, other
+ * texts the opposite; this library says P_tgt (target) and Q_dft (draft).
+ *
+ * General rules
+ *   - Plain C ABI.  Pointers are HOST pointers unless the name ends in _device /
+ *     the comment says "device".  No call allocates device memory: the KV cache
+ *     and the workspace are the caller's, borrowed until pass_destroy.
+ *   - Every call returns PASS_OK (0) or a negative PASS_ERR_*.  Nothing throws,
+ *     aborts or traps.  On error the state of every sequence is unchanged
+ *     (except after PASS_ERR_CUDA, where the CUDA context decides).
+ *   - All work is enqueued on the stream given to pass_create.  Calls are not
+ *     thread-safe per context.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef PASS_B200_H
+#define PASS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PASS_OK                 0
+#define PASS_ERR_INVALID_ARG   -1   /* NULL pointer, bad shape, k out of range, bad token id ... */
+#define PASS_ERR_CAPACITY      -2   /* KV capacity, workspace size or row limit exceeded */
+#define PASS_ERR_STATE         -3   /* e.g. pass_step before pass_prefill / pass_load_weights */
+#define PASS_ERR_CUDA          -4   /* a CUDA runtime or driver call failed */
+#define PASS_ERR_NONFINITE     -5   /* a non-finite logit reached the verify kernel */
+#define PASS_ERR_TIMEOUT       -6   /* a bounded device-side wait ran out */
+
+#define PASS_MAX_LOOKAHEAD     8    /* upper limit of k_max */
+#define PASS_MAX_ROWS        128    /* rows of one forward call: batch * (1 + 2k) <= 128 */
+
+#define PASS_DTYPE_FP32        0
+#define PASS_DTYPE_BF16        1
+
+typedef struct pass_ctx pass_ctx;   /* opaque */
+
+/* Shape of a LLaMA-style decoder (pre-norm, RMSNorm, rotary positions on adjacent
+ * pairs, SwiGLU, no biases, n_kv_heads == n_heads, untied output head): the
+ * paper's experiments use a re-implementation of the 7B LLaMA model. */
+typedef struct {
+    int n_layers, d_model, n_heads, d_head, d_ffn, vocab;
+    int k_max;        /* rows of the look-ahead embedding table, 1..PASS_MAX_LOOKAHEAD */
+    int max_batch;    /* independent sequences held by the context */
+    int kv_capacity;  /* positions per sequence */
+    int dtype;        /* PASS_DTYPE_*: type of weights AND of the KV cache */
+    float rms_eps, rope_theta;
+} pass_config;
+
+/* Device pointers to the weights, canonical [out_features, in_features] row-major,
+ * all of type cfg.dtype.  Per-layer entries are HOST arrays of n_layers device pointers.
+ * la_emb is the [k_max, d_model] look-ahead table ("Look-ahead embeddings":
+ * L extra INPUT embeddings; the output dictionary is unchanged). */
+typedef struct {
+    const void *tok_emb;      /* [vocab, d_model] */
+    const void *la_emb;       /* [k_max, d_model] */
+    const void *lm_head;      /* [vocab, d_model] */
+    const void *final_norm;   /* [d_model] */
+    const void *const *wq, *const *wk, *const *wv, *const *wo;   /* [d_model, d_model] */
+    const void *const *wg, *const *wu;                            /* [d_ffn, d_model] */
+    const void *const *wd;                                        /* [d_model, d_ffn] */
+    const void *const *norm_attn, *const *norm_ffn;               /* [d_model] */
+} pass_weights;
+
+/* Bytes the caller must provide.  kv: EACH of kv_k and kv_v.  Returns 0 on a bad config. */
+size_t pass_kv_bytes(const pass_config *cfg);
+size_t pass_workspace_bytes(const pass_config *cfg);
+
+/*
+ * Create a context on the current CUDA device.
+ *   kv_k_device, kv_v_device : caller-allocated device buffers of pass_kv_bytes() each,
+ *                              256-byte aligned; layout is private to the library.
+ *   workspace_device         : caller-allocated, pass_workspace_bytes(), 256-byte aligned.
+ *   cuda_stream              : a cudaStream_t (NULL = default stream).
+ * The buffers are borrowed until pass_destroy; the library never frees them.
+ * Errors: INVALID_ARG (NULL, misaligned, unsupported shape: d_model != n_heads*d_head,
+ * d_head not 64 or 128, k_max out of range), CAPACITY (buffers too small), CUDA.
+ */
+int pass_create(const pass_config *cfg, void *kv_k_device, void *kv_v_device, size_t kv_bytes,
+                void *workspace_device, size_t workspace_bytes, void *cuda_stream,
+                pass_ctx **out);
+
+/* Borrow the weights (device memory, unchanged and alive until pass_destroy).
+ * Builds the TMA descriptors of the weight-streaming GEMMs.  Errors: INVALID_ARG
+ * (NULL or misaligned pointer: every matrix must be 16-byte aligned), CUDA. */
+int pass_load_weights(pass_ctx *ctx, const pass_weights *w);
+
+/*
+ * Prompt processing for sequence `seq` (Algorithm 1: "initial prompt sequence
+ * x_0..x_t; n <- t").  Caches K/V of tokens[0..n-2]; tokens[n-1] becomes the pending
+ * token that the first pass_step feeds; pending drafts are dropped.  n >= 1.
+ * Resets the sequence first.  Synchronises the stream.
+ * Errors: INVALID_ARG (bad seq, n < 1, id outside [0, vocab)), CAPACITY (n-1 > kv_capacity),
+ * STATE (weights not loaded), CUDA.
+ */
+int pass_prefill(pass_ctx *ctx, int seq, const int32_t *tokens, int n);
+
+/*
+ * One PaSS iteration for ALL max_batch sequences (each must have been prefilled).
+ * Per sequence, with m in {0, k} pending drafts d_1..d_m drawn from laws Q_dft,1..m:
+ *   rows  [pending, d_1..d_m, LA_1..LA_k] (padded to 1+2k rows) at positions len, len+1, ...
+ *   P_tgt,j = softmax(logits_j / T) for j = 0..m          (validation phase of Algorithm 1)
+ *   draft j is accepted iff u[j-1] < min(1, P_tgt,j-1[d_j] / Q_dft,j[d_j])   (strict <)
+ *   first rejection at j: final token y ~ norm(max(0, P_tgt,j-1 - Q_dft,j)) and stop;
+ *   no rejection:         final token y ~ P_tgt,m  ("sample extra token")
+ *   emitted tokens = accepted drafts then y; len += number emitted; pending = y
+ *   if no draft was rejected the k rows after them give the next drafts
+ *   d'_t ~ Q'_t = softmax(logits_{m+t} / T) (drafting phase), else the next call has m = 0.
+ * temperature == 0 means greedy (one-hot laws at the first argmax).
+ * Sampling y ~ w uses inverse CDF in vocabulary order: smallest i with
+ * w_0 + .. + w_i > u * sum(w).  All of this is computed in float64 on the device.
+ *
+ *   k_lookahead : 0..k_max.  k = 0 is the auto-regressive baseline (one row, one token).
+ *   uniforms    : [max_batch][2k+1] floats in [0,1).  Slot j-1 (j=1..k): accept test of
+ *                 draft j; slot k: the final token; slot k+t (t=1..k): next draft t.
+ *                 May be NULL iff temperature == 0.
+ *   out_tokens  : [max_batch][k_max+1] int32, the emitted tokens of each sequence.
+ *   n_out       : [max_batch] int32, how many were emitted: 1 .. k+1 (every call adds at
+ *                 least one token - section "Parallel Speculative Sampling").
+ * Changing k_lookahead or temperature between calls drops pending drafts (they were
+ * drawn under other settings).  The step runs as one CUDA graph; the call copies the
+ * uniforms in, launches, copies the result out and synchronises the stream.
+ * Errors: INVALID_ARG, CAPACITY (len + 1 + 2k > kv_capacity for some sequence, or
+ * max_batch*(1+2k) > PASS_MAX_ROWS), STATE, NONFINITE, TIMEOUT, CUDA.
+ */
+int pass_step(pass_ctx *ctx, int k_lookahead, float temperature, const float *uniforms,
+              int32_t *out_tokens, int32_t *n_out);
+
+/*
+ * The same iteration without host round trip: reads the uniforms from DEVICE memory
+ * (same layout, may be NULL iff temperature == 0), enqueues the step and returns at once.
+ * Results stay on the device until pass_step_collect.  Capacity is checked against an
+ * upper bound of each sequence's length (k+1 tokens per uncollected step).
+ */
+int pass_step_enqueue(pass_ctx *ctx, int k_lookahead, float temperature,
+                      const float *uniforms_device);
+/* Synchronise and fetch the LAST enqueued step's result (same meaning as in pass_step). */
+int pass_step_collect(pass_ctx *ctx, int32_t *out_tokens, int32_t *n_out);
+
+/*
+ * Multi-token forward for one sequence: n rows appended at positions len .. len+n-1
+ * ("a single forward pass on n tokens in parallel").  ids in [0, vocab) are vocabulary
+ * tokens; id = vocab + j (0 <= j < k_max) feeds look-ahead embedding j as an input row.
+ *   logits_out_device : [n][vocab] float32 on the device, or NULL.
+ *   commit            : rows whose K/V are kept, 0..n; len += commit.  Rows after them
+ *                       are dead (overwritten by the next call).
+ * Drops pending drafts of the sequence; the pending token is left alone.
+ * 1 <= n <= PASS_MAX_ROWS.  Synchronises the stream.
+ * Errors: INVALID_ARG, CAPACITY (len + n > kv_capacity), STATE, CUDA.
+ */
+int pass_forward_tokens(pass_ctx *ctx, int seq, const int32_t *tokens, int n,
+                        float *logits_out_device, int commit);
+
+/* Forget everything about sequence `seq` (len = 0, no pending token, no drafts). */
+int pass_reset(pass_ctx *ctx, int seq);
+
+/*
+ * Restore cached keys/values of one layer (e.g. from a saved session): n positions from
+ * pos0, k and v as HOST arrays [n][d_model] in cfg.dtype, keys already rotated.  Does not
+ * change len; call pass_set_state afterwards.  Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+int pass_set_kv(pass_ctx *ctx, int seq, int layer, int pos0, int n, const void *k, const void *v);
+/* Read back cached keys/values of one layer, same layout (for inspection and tests). */
+int pass_get_kv(pass_ctx *ctx, int seq, int layer, int pos0, int n, void *k, void *v);
+/* Set len and the pending token of a sequence directly; drops pending drafts. */
+int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
+
+/* pass_get_debug selectors.  Each copies to a HOST buffer and synchronises. */
+#define PASS_DBG_LOGITS        0  /* float32 [rows][vocab] of the last forward (rows = B*(1+2k)) */
+#define PASS_DBG_DRAFT_LOGITS  1  /* float32 [max_batch][k_max][vocab]: logits the pending drafts were drawn from */
+#define PASS_DBG_KV_LEN        2  /* int32 [max_batch] */
+#define PASS_DBG_N_DRAFT       3  /* int32 [max_batch]: m */
+#define PASS_DBG_DRAFTS        4  /* int32 [max_batch][k_max] */
+#define PASS_DBG_PENDING       5  /* int32 [max_batch] */
+#define PASS_DBG_N_ACCEPTED    6  /* int32 [max_batch]: accepted drafts of the last step */
+#define PASS_DBG_STATUS        7  /* int32 [1]: device status word (0 = fine) */
+#define PASS_DBG_HIDDEN        8  /* float32 [rows][d_model]: residual stream after the last layer */
+int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
+
+/* Number of kernel launches (graph nodes) of the last pass_step / pass_step_enqueue. */
+int pass_last_step_launches(pass_ctx *ctx);
+/* Stream of the context (a cudaStream_t), so that callers can time on it. */
+void *pass_stream(pass_ctx *ctx);
+
+void pass_destroy(pass_ctx *ctx);
+const char *pass_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PASS_B200_H */
