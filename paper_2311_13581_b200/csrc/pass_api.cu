@@ -1,0 +1,654 @@
+// C-ABI entry points of the PaSS step library: context, workspace carving, the forward
+// schedule, CUDA-graph capture of the step, and the host mirror of the sequence state.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "kernels_simt.cuh"
+#include "kernels_verify.cuh"
+
+using namespace pass;
+
+namespace {
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        const size_t o = off;
+        off += (bytes + 255) & ~(size_t)255;
+        return o;
+    }
+};
+
+struct Layout {
+    size_t states, params, unif, status, row_seq, row_pos, tok, cs, invfreq;
+    size_t h, xn, qkv, attn, gu, act, logits;
+    size_t E, chunk, row_sum, row_max, amax_val, amax_idx, q_logits, q_E, q_sum, scratch;
+    size_t total;
+};
+
+bool config_ok(const pass_config* c) {
+    if (!c) return false;
+    if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ffn < 8 || c->vocab < 2) return false;
+    if (c->d_head != 64 && c->d_head != 128) return false;
+    if ((long long)c->n_heads * c->d_head != c->d_model) return false;
+    if (c->d_model % 8 || c->d_ffn % 8) return false;
+    if (c->k_max < 1 || c->k_max > kMaxLA) return false;
+    if (c->max_batch < 1 || c->max_batch > kMaxRows) return false;
+    if (c->kv_capacity < 1) return false;
+    if (c->dtype != PASS_DTYPE_FP32 && c->dtype != PASS_DTYPE_BF16) return false;
+    if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+    return true;
+}
+
+size_t esize(int dtype) { return dtype == PASS_DTYPE_FP32 ? 4 : 2; }
+
+Layout make_layout(const pass_config& c) {
+    Layout L;
+    Carve cv;
+    const size_t R = kMaxRows, d = c.d_model, f = c.d_ffn, V = c.vocab, B = c.max_batch;
+    L.states = cv.take(B * sizeof(SeqState));
+    L.params = cv.take(sizeof(StepParams));
+    L.unif = cv.take(B * kUSlots * sizeof(float));
+    L.status = cv.take(sizeof(int));
+    L.row_seq = cv.take(R * sizeof(int));
+    L.row_pos = cv.take(R * sizeof(int));
+    L.tok = cv.take(R * sizeof(int));
+    L.cs = cv.take(R * (c.d_head / 2) * sizeof(float2));
+    L.invfreq = cv.take((c.d_head / 2) * sizeof(double));
+    L.h = cv.take(R * d * 4);
+    L.xn = cv.take(R * d * 4);
+    L.qkv = cv.take(R * 3 * d * 4);
+    L.attn = cv.take(R * d * 4);
+    L.gu = cv.take(R * 2 * f * 4);
+    L.act = cv.take(R * f * 4);
+    L.logits = cv.take(R * V * 4);
+    L.E = cv.take(R * V * 8);
+    L.chunk = cv.take(R * kChunks * 8);
+    L.row_sum = cv.take(R * kVerifySplits * 8);
+    L.row_max = cv.take(R * 4);
+    L.amax_val = cv.take(R * kVerifySplits * 4);
+    L.amax_idx = cv.take(R * kVerifySplits * 4);
+    L.q_logits = cv.take(B * 2 * c.k_max * V * 4);
+    L.q_E = cv.take(B * 2 * c.k_max * V * 8);
+    L.q_sum = cv.take(B * 2 * c.k_max * kVerifySplits * 8);
+    L.scratch = cv.take(B * kChunks * 8);
+    L.total = cv.off;
+    return L;
+}
+
+constexpr int kParamRing = 64;
+
+}  // namespace
+
+struct pass_ctx {
+    pass_config cfg;
+    ModelDims md;
+    cudaStream_t stream;
+    void *kv_k, *kv_v;
+    char* ws;
+    Layout L;
+    // carved pointers
+    SeqState* d_states;
+    StepParams* d_params;
+    float* d_unif;
+    int *d_status, *d_row_seq, *d_row_pos, *d_tok;
+    float2* d_cs;
+    double* d_invfreq;
+    float *d_h, *d_xn, *d_qkv, *d_attn, *d_gu, *d_act, *d_logits;
+    VerifyBufs vb;
+    double* d_scratch;
+    // weights
+    bool weights_loaded = false;
+    const void *tok_emb, *la_emb, *lm_head, *final_norm;
+    std::vector<const void*> wq, wk, wv, wo, wg, wu, wd, norm_attn, norm_ffn;
+    // host mirror
+    std::vector<int> len_ub;
+    std::vector<char> prefilled;
+    bool have_last = false, params_on_device = false;
+    int last_k = -1;
+    float last_T = -1.f;
+    int dev_drop = 0;
+    bool pending_collect = false;
+    int last_rows = 0;
+    // pinned staging
+    StepParams* pin_params = nullptr;   // ring
+    int ring_pos = 0;
+    float* pin_unif = nullptr;
+    SeqState* pin_states = nullptr;
+    int* pin_status = nullptr;
+    int* pin_tok = nullptr;
+    // graphs
+    std::map<int, cudaGraphExec_t> graphs;
+    std::map<int, int> graph_launches;
+    bool use_graph = true;
+    int launches = 0, last_step_launches = 0;
+};
+
+#define CUDA_TRY(expr)                                                                     \
+    do {                                                                                   \
+        cudaError_t e_ = (expr);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            if (getenv("PASS_LOG")) fprintf(stderr, "[pass] %s failed: %s (%s:%d)\n", #expr, \
+                                            cudaGetErrorString(e_), __FILE__, __LINE__);   \
+            return PASS_ERR_CUDA;                                                          \
+        }                                                                                  \
+    } while (0)
+
+#define LAUNCH(ctx, kern, grid, block, ...)                           \
+    do {                                                              \
+        kern<<<(grid), (block), 0, (ctx)->stream>>>(__VA_ARGS__);     \
+        (ctx)->launches++;                                            \
+    } while (0)
+
+// ------------------------------------------------------------------------------- small kernels
+__global__ void k_update_state(SeqState* states, int seq, int set_len, int len, int add_len,
+                               int set_pending, int pending, int clear_all) {
+    SeqState& st = states[seq];
+    if (clear_all) {
+        st.kv_len = 0; st.pending = 0; st.has_pending = 0; st.m = 0; st.q_sel = 0;
+        st.n_out = 0; st.n_acc = 0;
+    }
+    if (set_len) st.kv_len = len;
+    st.kv_len += add_len;
+    if (set_pending) { st.pending = pending; st.has_pending = 1; }
+    st.m = 0;
+}
+
+// Between the caller's [n][d_model] layout and the cache's [head][position][d_head].
+template <typename KVT>
+__global__ void k_kv_scatter(const KVT* __restrict__ src, ModelDims md, int layer, int seq, int pos0,
+                             int n, KVT* __restrict__ cache, int gather) {
+    const size_t total = (size_t)n * md.d;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int p = (int)(i / md.d), c = (int)(i % md.d);
+        const size_t o = kv_index(md, layer, seq, c / md.dh, pos0 + p) + c % md.dh;
+        if (gather) const_cast<KVT*>(src)[i] = cache[o];
+        else cache[o] = src[i];
+    }
+}
+
+// ------------------------------------------------------------------------------- forward
+template <typename WT>
+static void enqueue_layers(pass_ctx* c, int R) {
+    const ModelDims& md = c->md;
+    const int d = md.d, f = md.f;
+    const WT* dummy = nullptr;
+    (void)dummy;
+    LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
+    const int gw = 8;   // warps (features) per GEMM block
+    for (int l = 0; l < md.n_layers; l++) {
+        LAUNCH(c, (k_rmsnorm<WT>), R, 256, c->d_h, (const WT*)c->norm_attn[l], d, md.eps, c->d_xn);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wq[l], d, d, R, c->d_qkv, 3 * d, 0);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wk[l], d, d, R, c->d_qkv + d, 3 * d, 0);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wv[l], d, d, R, c->d_qkv + 2 * d, 3 * d, 0);
+        LAUNCH(c, (k_rope_kv<WT>), R, 256, c->d_qkv, c->d_cs, c->d_row_seq, c->d_row_pos, md, l, (WT*)c->kv_k, (WT*)c->kv_v);
+        if (md.dh == 128)
+            LAUNCH(c, (k_attn_simple<WT, 128>), dim3(md.H, R), 128, c->d_qkv, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, c->d_attn);
+        else
+            LAUNCH(c, (k_attn_simple<WT, 64>), dim3(md.H, R), 128, c->d_qkv, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, c->d_attn);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_attn, d, (const WT*)c->wo[l], d, d, R, c->d_h, d, 1);
+        LAUNCH(c, (k_rmsnorm<WT>), R, 256, c->d_h, (const WT*)c->norm_ffn[l], d, md.eps, c->d_xn);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (f + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wg[l], f, d, R, c->d_gu, 2 * f, 0);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (f + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wu[l], f, d, R, c->d_gu + f, 2 * f, 0);
+        LAUNCH(c, k_swiglu, dim3((f + 255) / 256, R), 256, c->d_gu, f, c->d_act);
+        LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_act, f, (const WT*)c->wd[l], d, f, R, c->d_h, d, 1);
+    }
+}
+
+template <typename WT>
+static void enqueue_head(pass_ctx* c, int R) {
+    const ModelDims& md = c->md;
+    const int gw = 8;
+    LAUNCH(c, (k_rmsnorm<WT>), R, 256, c->d_h, (const WT*)c->final_norm, md.d, md.eps, c->d_xn);
+    LAUNCH(c, (k_gemm_simt<WT, 16>), (md.V + gw - 1) / gw, gw * 32, c->d_xn, md.d, (const WT*)c->lm_head, md.V, md.d, R, c->d_logits, md.V, 0);
+}
+
+template <typename WT>
+static void enqueue_step(pass_ctx* c, int k) {
+    const ModelDims& md = c->md;
+    const int M = 1 + 2 * k, R = md.B * M;
+    LAUNCH(c, (k_assemble_step<WT>), R, 256, (const WT*)c->tok_emb, (const WT*)c->la_emb, c->d_states,
+           c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos);
+    enqueue_layers<WT>(c, R);
+    enqueue_head<WT>(c, R);
+    LAUNCH(c, k_verify_stats, dim3(R, kVerifySplits), kVerifyThreads, c->vb, c->d_states, c->d_params, M, md.V, md.k_max);
+    LAUNCH(c, k_verify_decide, md.B, 1024, c->vb, c->d_states, c->d_params, c->d_unif, M, md.V, md.k_max, c->d_scratch);
+}
+
+static void enqueue_step_any(pass_ctx* c, int k) {
+    if (c->md.dtype == PASS_DTYPE_FP32) enqueue_step<float>(c, k);
+    else enqueue_step<__nv_bfloat16>(c, k);
+}
+
+static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool want_logits) {
+    memcpy(c->pin_tok, tokens, sizeof(int) * n);
+    CUDA_TRY(cudaMemcpyAsync(c->d_tok, c->pin_tok, sizeof(int) * n, cudaMemcpyHostToDevice, c->stream));
+    if (c->md.dtype == PASS_DTYPE_FP32) {
+        LAUNCH(c, (k_assemble_tokens<float>), n, 256, (const float*)c->tok_emb, (const float*)c->la_emb,
+               c->d_states, c->d_tok, seq, c->md.d, c->md.V, c->d_h, c->d_row_seq, c->d_row_pos);
+        enqueue_layers<float>(c, n);
+        if (want_logits) enqueue_head<float>(c, n);
+    } else {
+        LAUNCH(c, (k_assemble_tokens<__nv_bfloat16>), n, 256, (const __nv_bfloat16*)c->tok_emb,
+               (const __nv_bfloat16*)c->la_emb, c->d_states, c->d_tok, seq, c->md.d, c->md.V, c->d_h,
+               c->d_row_seq, c->d_row_pos);
+        enqueue_layers<__nv_bfloat16>(c, n);
+        if (want_logits) enqueue_head<__nv_bfloat16>(c, n);
+    }
+    c->last_rows = n;
+    CUDA_TRY(cudaGetLastError());
+    return PASS_OK;
+}
+
+// ------------------------------------------------------------------------------- C ABI
+extern "C" {
+
+size_t pass_kv_bytes(const pass_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return (size_t)cfg->n_layers * cfg->max_batch * cfg->kv_capacity * cfg->d_model * esize(cfg->dtype);
+}
+
+size_t pass_workspace_bytes(const pass_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return make_layout(*cfg).total;
+}
+
+int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes, void* workspace,
+                size_t workspace_bytes, void* cuda_stream, pass_ctx** out) {
+    if (!out) return PASS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg) || !kv_k || !kv_v || !workspace) return PASS_ERR_INVALID_ARG;
+    if (((uintptr_t)kv_k | (uintptr_t)kv_v | (uintptr_t)workspace) & 255) return PASS_ERR_INVALID_ARG;
+    if (kv_bytes < pass_kv_bytes(cfg)) return PASS_ERR_CAPACITY;
+    const Layout L = make_layout(*cfg);
+    if (workspace_bytes < L.total) return PASS_ERR_CAPACITY;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return PASS_ERR_CUDA;
+    pass_ctx* c = new (std::nothrow) pass_ctx();
+    if (!c) return PASS_ERR_CUDA;
+    c->cfg = *cfg;
+    c->md = ModelDims{cfg->n_layers, cfg->d_model, cfg->n_heads, cfg->d_head, cfg->d_ffn, cfg->vocab,
+                      cfg->k_max, cfg->max_batch, cfg->kv_capacity, cfg->dtype, cfg->rms_eps,
+                      cfg->rope_theta};
+    c->stream = (cudaStream_t)cuda_stream;
+    c->kv_k = kv_k;
+    c->kv_v = kv_v;
+    c->ws = (char*)workspace;
+    c->L = L;
+    char* w = c->ws;
+    c->d_states = (SeqState*)(w + L.states);
+    c->d_params = (StepParams*)(w + L.params);
+    c->d_unif = (float*)(w + L.unif);
+    c->d_status = (int*)(w + L.status);
+    c->d_row_seq = (int*)(w + L.row_seq);
+    c->d_row_pos = (int*)(w + L.row_pos);
+    c->d_tok = (int*)(w + L.tok);
+    c->d_cs = (float2*)(w + L.cs);
+    c->d_invfreq = (double*)(w + L.invfreq);
+    c->d_h = (float*)(w + L.h);
+    c->d_xn = (float*)(w + L.xn);
+    c->d_qkv = (float*)(w + L.qkv);
+    c->d_attn = (float*)(w + L.attn);
+    c->d_gu = (float*)(w + L.gu);
+    c->d_act = (float*)(w + L.act);
+    c->d_logits = (float*)(w + L.logits);
+    c->vb.logits = c->d_logits;
+    c->vb.E = (double*)(w + L.E);
+    c->vb.chunk = (double*)(w + L.chunk);
+    c->vb.row_sum = (double*)(w + L.row_sum);
+    c->vb.row_max = (float*)(w + L.row_max);
+    c->vb.amax_val = (float*)(w + L.amax_val);
+    c->vb.amax_idx = (int*)(w + L.amax_idx);
+    c->vb.q_logits = (float*)(w + L.q_logits);
+    c->vb.q_E = (double*)(w + L.q_E);
+    c->vb.q_sum = (double*)(w + L.q_sum);
+    c->vb.status = c->d_status;
+    c->d_scratch = (double*)(w + L.scratch);
+    c->len_ub.assign(cfg->max_batch, 0);
+    c->prefilled.assign(cfg->max_batch, 0);
+    c->use_graph = getenv("PASS_NO_GRAPH") == nullptr;
+
+    auto fail = [&](int code) { pass_destroy(c); return code; };
+    if (cudaMallocHost((void**)&c->pin_params, sizeof(StepParams) * kParamRing) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaMallocHost((void**)&c->pin_unif, sizeof(float) * cfg->max_batch * kUSlots) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaMallocHost((void**)&c->pin_states, sizeof(SeqState) * cfg->max_batch) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaMallocHost((void**)&c->pin_status, sizeof(int)) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaMallocHost((void**)&c->pin_tok, sizeof(int) * kMaxRows) != cudaSuccess) return fail(PASS_ERR_CUDA);
+
+    // zero the small state region; rotary frequencies theta^(-2i/d_head) in float64
+    if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    std::vector<double> inv(cfg->d_head / 2);
+    for (int i = 0; i < cfg->d_head / 2; i++)
+        inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
+    if (cudaMemcpyAsync(c->d_invfreq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    *out = c;
+    return PASS_OK;
+}
+
+int pass_load_weights(pass_ctx* c, const pass_weights* w) {
+    if (!c || !w) return PASS_ERR_INVALID_ARG;
+    const void* singles[] = {w->tok_emb, w->la_emb, w->lm_head, w->final_norm};
+    for (const void* p : singles)
+        if (!p || ((uintptr_t)p & 15)) return PASS_ERR_INVALID_ARG;
+    const void* const* arrays[] = {w->wq, w->wk, w->wv, w->wo, w->wg, w->wu, w->wd, w->norm_attn, w->norm_ffn};
+    for (auto a : arrays) {
+        if (!a) return PASS_ERR_INVALID_ARG;
+        for (int l = 0; l < c->md.n_layers; l++)
+            if (!a[l] || ((uintptr_t)a[l] & 15)) return PASS_ERR_INVALID_ARG;
+    }
+    c->tok_emb = w->tok_emb; c->la_emb = w->la_emb; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
+    const int nl = c->md.n_layers;
+    c->wq.assign(w->wq, w->wq + nl); c->wk.assign(w->wk, w->wk + nl); c->wv.assign(w->wv, w->wv + nl);
+    c->wo.assign(w->wo, w->wo + nl); c->wg.assign(w->wg, w->wg + nl); c->wu.assign(w->wu, w->wu + nl);
+    c->wd.assign(w->wd, w->wd + nl);
+    c->norm_attn.assign(w->norm_attn, w->norm_attn + nl);
+    c->norm_ffn.assign(w->norm_ffn, w->norm_ffn + nl);
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+    c->graphs.clear();
+    c->weights_loaded = true;
+    return PASS_OK;
+}
+
+int pass_reset(pass_ctx* c, int seq) {
+    if (!c || seq < 0 || seq >= c->md.B) return PASS_ERR_INVALID_ARG;
+    LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, 0, 0, 0, 1);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->len_ub[seq] = 0;
+    c->prefilled[seq] = 0;
+    return PASS_OK;
+}
+
+int pass_set_state(pass_ctx* c, int seq, int len, int32_t pending) {
+    if (!c || seq < 0 || seq >= c->md.B || len < 0 || pending < 0 || pending >= c->md.V) return PASS_ERR_INVALID_ARG;
+    if (len > c->md.cap) return PASS_ERR_CAPACITY;
+    LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 1, len, 0, 1, (int)pending, 0);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->len_ub[seq] = len;
+    c->prefilled[seq] = 1;
+    return PASS_OK;
+}
+
+int pass_forward_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, float* logits_out_device,
+                        int commit) {
+    if (!c || !tokens || seq < 0 || seq >= c->md.B || n < 1 || n > kMaxRows || commit < 0 || commit > n)
+        return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded) return PASS_ERR_STATE;
+    for (int i = 0; i < n; i++)
+        if (tokens[i] < 0 || tokens[i] >= c->md.V + c->md.k_max) return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    if (c->len_ub[seq] + n > c->md.cap) return PASS_ERR_CAPACITY;
+    int rc = run_tokens(c, seq, tokens, n, logits_out_device != nullptr);
+    if (rc != PASS_OK) return rc;
+    if (logits_out_device)
+        CUDA_TRY(cudaMemcpyAsync(logits_out_device, c->d_logits, sizeof(float) * (size_t)n * c->md.V,
+                                 cudaMemcpyDeviceToDevice, c->stream));
+    LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, commit, 0, 0, 0);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->len_ub[seq] += commit;
+    return PASS_OK;
+}
+
+int pass_prefill(pass_ctx* c, int seq, const int32_t* tokens, int n) {
+    if (!c || !tokens || seq < 0 || seq >= c->md.B || n < 1) return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded) return PASS_ERR_STATE;
+    for (int i = 0; i < n; i++)
+        if (tokens[i] < 0 || tokens[i] >= c->md.V) return PASS_ERR_INVALID_ARG;
+    if (n - 1 > c->md.cap) return PASS_ERR_CAPACITY;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    int rc = pass_reset(c, seq);
+    if (rc != PASS_OK) return rc;
+    for (int s = 0; s < n - 1; s += kMaxRows) {
+        const int rows = std::min(kMaxRows, n - 1 - s);
+        rc = run_tokens(c, seq, tokens + s, rows, false);
+        if (rc != PASS_OK) return rc;
+        LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, rows, 0, 0, 0);
+        CUDA_TRY(cudaStreamSynchronize(c->stream));   // pin_tok is reused by the next chunk
+    }
+    LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, 0, 1, (int)tokens[n - 1], 0);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->len_ub[seq] = n - 1;
+    c->prefilled[seq] = 1;
+    return PASS_OK;
+}
+
+static int step_checks(pass_ctx* c, int k, float T, const void* uniforms) {
+    if (!c || k < 0 || k > c->md.k_max || !(T >= 0.f) || !std::isfinite(T)) return PASS_ERR_INVALID_ARG;
+    if (!uniforms && T != 0.f) return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded) return PASS_ERR_STATE;
+    if (c->md.B * (1 + 2 * k) > kMaxRows) return PASS_ERR_CAPACITY;
+    for (int b = 0; b < c->md.B; b++) {
+        if (!c->prefilled[b]) return PASS_ERR_STATE;
+        if (c->len_ub[b] + 1 + 2 * k > c->md.cap) return PASS_ERR_CAPACITY;
+    }
+    return PASS_OK;
+}
+
+static int step_launch(pass_ctx* c, int k, float T) {
+    // step parameters: only re-sent when they differ from what the device holds
+    const int drop = (c->have_last && (k != c->last_k || T != c->last_T)) ? 1 : 0;
+    if (!c->params_on_device || !c->have_last || k != c->last_k || T != c->last_T || drop != c->dev_drop) {
+        if (c->ring_pos == kParamRing) {
+            CUDA_TRY(cudaStreamSynchronize(c->stream));
+            c->ring_pos = 0;
+        }
+        StepParams* p = c->pin_params + c->ring_pos++;
+        p->temperature = T; p->k = k; p->drop_drafts = drop; p->pad_ = 0;
+        CUDA_TRY(cudaMemcpyAsync(c->d_params, p, sizeof(StepParams), cudaMemcpyHostToDevice, c->stream));
+        c->params_on_device = true;
+        c->dev_drop = drop;
+    }
+    c->have_last = true; c->last_k = k; c->last_T = T;
+    c->launches = 0;
+    if (c->use_graph) {
+        auto it = c->graphs.find(k);
+        if (it == c->graphs.end()) {
+            cudaGraph_t g = nullptr;
+            CUDA_TRY(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+            enqueue_step_any(c, k);
+            cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+            if (e != cudaSuccess || !g) return PASS_ERR_CUDA;
+            cudaGraphExec_t ge = nullptr;
+            e = cudaGraphInstantiate(&ge, g, 0);
+            cudaGraphDestroy(g);
+            if (e != cudaSuccess) return PASS_ERR_CUDA;
+            c->graphs[k] = ge;
+            c->graph_launches[k] = c->launches;
+            it = c->graphs.find(k);
+        }
+        CUDA_TRY(cudaGraphLaunch(it->second, c->stream));
+        c->last_step_launches = c->graph_launches[k];
+    } else {
+        enqueue_step_any(c, k);
+        CUDA_TRY(cudaGetLastError());
+        c->last_step_launches = c->launches;
+    }
+    c->last_rows = c->md.B * (1 + 2 * k);
+    for (int b = 0; b < c->md.B; b++) c->len_ub[b] += k + 1;
+    c->pending_collect = true;
+    return PASS_OK;
+}
+
+int pass_step_enqueue(pass_ctx* c, int k, float T, const float* uniforms_device) {
+    int rc = step_checks(c, k, T, uniforms_device);
+    if (rc != PASS_OK) return rc;
+    if (uniforms_device)
+        CUDA_TRY(cudaMemcpy2DAsync(c->d_unif, kUSlots * sizeof(float), uniforms_device,
+                                   (2 * k + 1) * sizeof(float), (2 * k + 1) * sizeof(float), c->md.B,
+                                   cudaMemcpyDeviceToDevice, c->stream));
+    return step_launch(c, k, T);
+}
+
+int pass_step_collect(pass_ctx* c, int32_t* out_tokens, int32_t* n_out) {
+    if (!c) return PASS_ERR_INVALID_ARG;
+    if (!c->pending_collect) return PASS_ERR_STATE;
+    CUDA_TRY(cudaMemcpyAsync(c->pin_states, c->d_states, sizeof(SeqState) * c->md.B, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(cudaMemcpyAsync(c->pin_status, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    c->pending_collect = false;
+    for (int b = 0; b < c->md.B; b++) c->len_ub[b] = c->pin_states[b].kv_len;
+    const int status = *c->pin_status;
+    if (status != 0) {
+        CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream));
+        CUDA_TRY(cudaStreamSynchronize(c->stream));
+        if (status & kStatusTimeout) return PASS_ERR_TIMEOUT;
+        if (status & kStatusNonFinite) return PASS_ERR_NONFINITE;
+        return PASS_ERR_STATE;
+    }
+    for (int b = 0; b < c->md.B; b++) {
+        if (n_out) n_out[b] = c->pin_states[b].n_out;
+        if (out_tokens)
+            for (int j = 0; j <= c->md.k_max; j++)
+                out_tokens[b * (c->md.k_max + 1) + j] = j < c->pin_states[b].n_out ? c->pin_states[b].out_tokens[j] : -1;
+    }
+    return PASS_OK;
+}
+
+int pass_step(pass_ctx* c, int k, float T, const float* uniforms, int32_t* out_tokens, int32_t* n_out) {
+    if (!out_tokens || !n_out) return PASS_ERR_INVALID_ARG;
+    int rc = step_checks(c, k, T, uniforms);
+    if (rc != PASS_OK) return rc;
+    if (c->pending_collect) {
+        rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+        rc = step_checks(c, k, T, uniforms);
+        if (rc != PASS_OK) return rc;
+    }
+    if (uniforms) {
+        for (int b = 0; b < c->md.B; b++)
+            for (int j = 0; j < 2 * k + 1; j++) {
+                const float u = uniforms[b * (2 * k + 1) + j];
+                if (!(u >= 0.f && u < 1.f)) return PASS_ERR_INVALID_ARG;
+                c->pin_unif[b * kUSlots + j] = u;
+            }
+        CUDA_TRY(cudaMemcpyAsync(c->d_unif, c->pin_unif, sizeof(float) * c->md.B * kUSlots, cudaMemcpyHostToDevice, c->stream));
+    }
+    rc = step_launch(c, k, T);
+    if (rc != PASS_OK) return rc;
+    return pass_step_collect(c, out_tokens, n_out);
+}
+
+static int kv_copy(pass_ctx* c, int seq, int layer, int pos0, int n, void* k, void* v, int gather) {
+    if (!c || !k || !v || seq < 0 || seq >= c->md.B || layer < 0 || layer >= c->md.n_layers || pos0 < 0 || n < 1)
+        return PASS_ERR_INVALID_ARG;
+    if (pos0 + n > c->md.cap) return PASS_ERR_CAPACITY;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    const size_t es = esize(c->md.dtype), rowb = (size_t)c->md.d * es;
+    const size_t stage_bytes = (size_t)kMaxRows * c->md.V * 8;     // the E buffer doubles as staging
+    const int chunk = (int)std::max<size_t>(1, std::min<size_t>(n, stage_bytes / rowb));
+    void* stage = c->vb.E;
+    void* host[2] = {k, v};
+    void* cache[2] = {c->kv_k, c->kv_v};
+    for (int which = 0; which < 2; which++)
+        for (int s = 0; s < n; s += chunk) {
+            const int cn = std::min(chunk, n - s);
+            char* hp = (char*)host[which] + (size_t)s * rowb;
+            if (!gather) CUDA_TRY(cudaMemcpyAsync(stage, hp, cn * rowb, cudaMemcpyHostToDevice, c->stream));
+            const int blocks = (int)std::min<size_t>(1024, ((size_t)cn * c->md.d + 255) / 256);
+            if (es == 4)
+                LAUNCH(c, (k_kv_scatter<float>), blocks, 256, (const float*)stage, c->md, layer, seq, pos0 + s, cn, (float*)cache[which], gather);
+            else
+                LAUNCH(c, (k_kv_scatter<__nv_bfloat16>), blocks, 256, (const __nv_bfloat16*)stage, c->md, layer, seq, pos0 + s, cn, (__nv_bfloat16*)cache[which], gather);
+            if (gather) CUDA_TRY(cudaMemcpyAsync(hp, stage, cn * rowb, cudaMemcpyDeviceToHost, c->stream));
+            CUDA_TRY(cudaStreamSynchronize(c->stream));
+        }
+    CUDA_TRY(cudaGetLastError());
+    return PASS_OK;
+}
+
+int pass_set_kv(pass_ctx* c, int seq, int layer, int pos0, int n, const void* k, const void* v) {
+    return kv_copy(c, seq, layer, pos0, n, const_cast<void*>(k), const_cast<void*>(v), 0);
+}
+int pass_get_kv(pass_ctx* c, int seq, int layer, int pos0, int n, void* k, void* v) {
+    return kv_copy(c, seq, layer, pos0, n, k, v, 1);
+}
+
+int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
+    if (!c || !dst) return PASS_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    const int B = c->md.B, V = c->md.V, km = c->md.k_max;
+    auto need = [&](size_t n) { return bytes >= n; };
+    if (what == PASS_DBG_LOGITS || what == PASS_DBG_HIDDEN) {
+        const size_t n = (size_t)c->last_rows * (what == PASS_DBG_LOGITS ? V : c->md.d) * 4;
+        if (!need(n)) return PASS_ERR_CAPACITY;
+        CUDA_TRY(cudaMemcpy(dst, what == PASS_DBG_LOGITS ? c->d_logits : c->d_h, n, cudaMemcpyDeviceToHost));
+        return PASS_OK;
+    }
+    if (what == PASS_DBG_STATUS) {
+        if (!need(4)) return PASS_ERR_CAPACITY;
+        CUDA_TRY(cudaMemcpy(dst, c->d_status, 4, cudaMemcpyDeviceToHost));
+        return PASS_OK;
+    }
+    std::vector<SeqState> st(B);
+    CUDA_TRY(cudaMemcpy(st.data(), c->d_states, sizeof(SeqState) * B, cudaMemcpyDeviceToHost));
+    int* o = (int*)dst;
+    switch (what) {
+        case PASS_DBG_DRAFT_LOGITS: {
+            if (!need((size_t)B * km * V * 4)) return PASS_ERR_CAPACITY;
+            for (int b = 0; b < B; b++)
+                CUDA_TRY(cudaMemcpy((float*)dst + (size_t)b * km * V,
+                                    c->vb.q_logits + ((size_t)b * 2 + st[b].q_sel) * km * V,
+                                    (size_t)km * V * 4, cudaMemcpyDeviceToHost));
+            return PASS_OK;
+        }
+        case PASS_DBG_KV_LEN: if (!need(4 * B)) return PASS_ERR_CAPACITY; for (int b = 0; b < B; b++) o[b] = st[b].kv_len; return PASS_OK;
+        case PASS_DBG_N_DRAFT: if (!need(4 * B)) return PASS_ERR_CAPACITY; for (int b = 0; b < B; b++) o[b] = st[b].m; return PASS_OK;
+        case PASS_DBG_PENDING: if (!need(4 * B)) return PASS_ERR_CAPACITY; for (int b = 0; b < B; b++) o[b] = st[b].pending; return PASS_OK;
+        case PASS_DBG_N_ACCEPTED: if (!need(4 * B)) return PASS_ERR_CAPACITY; for (int b = 0; b < B; b++) o[b] = st[b].n_acc; return PASS_OK;
+        case PASS_DBG_DRAFTS:
+            if (!need((size_t)4 * B * km)) return PASS_ERR_CAPACITY;
+            for (int b = 0; b < B; b++)
+                for (int j = 0; j < km; j++) o[b * km + j] = j < st[b].m ? st[b].drafts[j] : -1;
+            return PASS_OK;
+        default: return PASS_ERR_INVALID_ARG;
+    }
+}
+
+int pass_last_step_launches(pass_ctx* c) { return c ? c->last_step_launches : 0; }
+void* pass_stream(pass_ctx* c) { return c ? (void*)c->stream : nullptr; }
+
+void pass_destroy(pass_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+    if (c->pin_params) cudaFreeHost(c->pin_params);
+    if (c->pin_unif) cudaFreeHost(c->pin_unif);
+    if (c->pin_states) cudaFreeHost(c->pin_states);
+    if (c->pin_status) cudaFreeHost(c->pin_status);
+    if (c->pin_tok) cudaFreeHost(c->pin_tok);
+    delete c;
+}
+
+const char* pass_strerror(int code) {
+    switch (code) {
+        case PASS_OK: return "ok";
+        case PASS_ERR_INVALID_ARG: return "invalid argument";
+        case PASS_ERR_CAPACITY: return "capacity exceeded (KV cache, workspace or row limit)";
+        case PASS_ERR_STATE: return "call not valid in this state";
+        case PASS_ERR_CUDA: return "CUDA call failed";
+        case PASS_ERR_NONFINITE: return "non-finite logit";
+        case PASS_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

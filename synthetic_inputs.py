@@ -155,3 +155,20 @@ def make_prompt(shape: ModelShape, length: int, seq: int = 0, seed: int = 0) -> 
 def step_uniforms(seed: int, seq: int, step: int, n_slots: int) -> torch.Tensor:
     """The uniforms of one PaSS step of one sequence: float32 [n_slots]."""
     return uniforms(seed, _S_UNIF + seq, step * 64, n_slots)
+
+
+_S_KV = 1 << 22
+
+
+def make_kv(shape: ModelShape, layer: int, n_pos: int, seq: int = 0, seed: int = 0, std: float = 1.0,
+            device="cpu"):
+    """Synthetic cached keys and values of one layer, [n_pos, d_model] each in the model dtype.
+
+    Stands in for the cache a long prompt would leave behind, so that long contexts can be
+    checked without paying for the prompt pass on the CPU side.
+    """
+    dt = _TORCH_DTYPE[shape.dtype]
+    base = _S_KV + (seq * 4096 + layer) * 2
+    k = normal(seed, base, n_pos * shape.d_model, std, device).view(n_pos, shape.d_model).to(dt)
+    v = normal(seed, base + 1, n_pos * shape.d_model, std, device).view(n_pos, shape.d_model).to(dt)
+    return k, v

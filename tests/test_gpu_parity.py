@@ -1,0 +1,215 @@
+"""Parity of the CUDA library with the CPU oracle, through the C ABI (needs a B200)."""
+import copy
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as si
+from oracle import pass_oracle as po
+
+pytestmark = pytest.mark.gpu
+
+TINY = si.SHAPES["tiny"]
+TINY_BF16 = dataclasses.replace(TINY, dtype="bf16")
+
+
+def _pb():
+    import paper_2311_13581_b200 as pb
+    return pb
+
+
+@pytest.fixture(scope="module")
+def tiny_w():
+    return si.make_weights(TINY, seed=0)
+
+
+def test_library_loaded_and_device_is_blackwell():
+    pb = _pb()
+    pb.load_library()
+    assert torch.cuda.is_available()
+    assert torch.cuda.get_device_capability(0)[0] == 10
+
+
+# ------------------------------------------------------------------ config 1: tiny fp32
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_tiny_fp32_lockstep_k2(tiny_w, T):
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY, 32)
+    ctx, oracles, _ = make_pair(TINY, 1, 32 + 64 + 3 * 8 + 8, [prompt], weights=tiny_w)
+    total, streams = 0, []
+    stats_all = None
+    step = 0
+    while total < 64:
+        stats, st = lockstep(ctx, oracles, 2, T, 4, step0=step)
+        step += 4
+        total += stats["tokens"]
+        streams += st[0]
+        assert stats["max_logit_err"] <= 1e-3, stats
+        stats_all = stats
+    if T == 0.0:
+        be = po.TransformerBackend(TINY, tiny_w, 32 + 96)
+        ar, _ = po.autoregressive(be, prompt, 0.0, 64, lambda i: 0.0)
+        assert streams[:64] == ar          # greedy PaSS == greedy auto-regressive, on the GPU
+    ctx.close()
+
+
+def test_tiny_fp32_multi_token_forward_equals_sequential_and_oracle(tiny_w):
+    pb = _pb()
+    prompt = si.make_prompt(TINY, 40)
+    ctx = pb.PassContext(TINY, si.weights_to(tiny_w, "cuda:0"), 1, 64)
+    ids = prompt[:13] + [TINY.vocab + 0, TINY.vocab + 1, TINY.vocab + 2]
+    z_all = ctx.forward_tokens(0, ids, commit=0).cpu().numpy()
+    rows = []
+    for t in ids:
+        rows.append(ctx.forward_tokens(0, [t], commit=1).cpu().numpy()[0])
+    z_seq = np.stack(rows)
+    assert np.max(np.abs(z_all - z_seq)) <= 2e-5
+    be = po.TransformerBackend(TINY, tiny_w, 64)
+    z_or = be.forward([("tok", t) for t in prompt[:13]] + [("la", 0), ("la", 1), ("la", 2)], 0)
+    assert np.max(np.abs(z_all - z_or)) <= 1e-3
+    assert np.max(np.abs(z_or)) > 0.1
+    # rollback: rows not committed are overwritten
+    ctx.reset(0)
+    ctx.forward_tokens(0, prompt[:5], commit=5, want_logits=False)
+    ctx.forward_tokens(0, [1, 2, 3], commit=0, want_logits=False)
+    z_b = ctx.forward_tokens(0, prompt[5:13], commit=8).cpu().numpy()
+    assert np.max(np.abs(z_b - z_or[5:13])) <= 1e-3
+    ctx.close()
+
+
+def test_prefill_cache_matches_oracle_cache(tiny_w):
+    pb = _pb()
+    prompt = si.make_prompt(TINY, 150)        # spans two 128-row chunks
+    ctx = pb.PassContext(TINY, si.weights_to(tiny_w, "cuda:0"), 2, 200)
+    ctx.prefill(1, prompt)
+    be = po.TransformerBackend(TINY, tiny_w, 200)
+    be.prefill(prompt[:-1])
+    for layer in range(TINY.n_layers):
+        k, v = ctx.get_kv(1, layer, 0, 149)
+        assert np.max(np.abs(k.double().numpy() - be.k[layer, :149])) <= 1e-4
+        assert np.max(np.abs(v.double().numpy() - be.v[layer, :149])) <= 1e-4
+    assert ctx.get_debug(pb.PASS_DBG_KV_LEN)[1] == 149
+    assert ctx.get_debug(pb.PASS_DBG_PENDING)[1] == prompt[-1]
+    ctx.close()
+
+
+def test_set_kv_round_trip(tiny_w):
+    pb = _pb()
+    ctx = pb.PassContext(TINY, si.weights_to(tiny_w, "cuda:0"), 2, 64)
+    k, v = si.make_kv(TINY, 1, 37, seq=1)
+    ctx.set_kv(1, 1, 5, k, v)
+    k2, v2 = ctx.get_kv(1, 1, 5, 37)
+    assert torch.equal(k, k2) and torch.equal(v, v2)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ batch, k sweep, bf16
+def test_tiny_fp32_batch3_ragged_lockstep(tiny_w):
+    from parity_util import lockstep, make_pair
+    prompts = [si.make_prompt(TINY, n, seq=b) for b, n in enumerate((32, 7, 19))]
+    ctx, oracles, _ = make_pair(TINY, 3, 128, prompts, weights=tiny_w)
+    stats, _ = lockstep(ctx, oracles, 2, 1.0, 12)
+    assert stats["max_logit_err"] <= 1e-3
+    assert stats["accepted"] > 0                     # multi-token steps did happen
+    lens = ctx.get_debug(_pb().PASS_DBG_KV_LEN)
+    assert len(set(lens.tolist())) == 3              # ragged
+    ctx.close()
+
+
+@pytest.mark.parametrize("k", [0, 1, 4, 8])
+def test_tiny_bf16_k_sweep_sampled(k):
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY_BF16, 24)
+    ctx, oracles, _ = make_pair(TINY_BF16, 1, 160, [prompt], seed=1)
+    stats, _ = lockstep(ctx, oracles, k, 0.8, 8, check_A=False)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
+def test_changing_k_and_temperature_between_steps(tiny_w):
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY, 16)
+    ctx, oracles, _ = make_pair(TINY, 1, 160, [prompt], weights=tiny_w)
+    step = 0
+    for k, T in ((2, 1.0), (4, 1.0), (4, 0.5), (1, 0.0), (3, 0.0), (2, 1.0)):
+        stats, _ = lockstep(ctx, oracles, k, T, 3, step0=step)
+        step += 3
+        assert stats["max_logit_err"] <= 1e-3
+    ctx.close()
+
+
+# ------------------------------------------------------------------ errors never fault
+def test_error_paths(tiny_w):
+    pb = _pb()
+    w = si.weights_to(tiny_w, "cuda:0")
+    ctx = pb.PassContext(TINY, w, 1, 48)
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(2, 0.0, None)                        # before prefill
+    assert e.value.code == -3
+    ctx.prefill(0, si.make_prompt(TINY, 8))
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(9, 0.0, None)                        # k > k_max
+    assert e.value.code == -1
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(2, 1.0, None)                        # NULL uniforms with T > 0
+    assert e.value.code == -1
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(2, 1.0, np.array([[0.1, 0.2, 1.0, 0.3, 0.4]], dtype=np.float32))   # u == 1
+    assert e.value.code == -1
+    with pytest.raises(pb.PassError) as e:
+        ctx.prefill(0, [TINY.vocab])                  # bad token id
+    assert e.value.code == -1
+    with pytest.raises(pb.PassError) as e:
+        ctx.prefill(0, list(range(60)))               # longer than the cache
+    assert e.value.code == -2
+    # capacity: len 7 + 1 + 2k > 48 once the sequence has grown
+    ctx.prefill(0, si.make_prompt(TINY, 8))
+    n = 0
+    with pytest.raises(pb.PassError) as e:
+        for _ in range(100):
+            ctx.step(8, 0.0, None)
+            n += 1
+    assert e.value.code == -2 and n > 5
+    ctx.close()
+
+
+def test_nonfinite_logits_are_reported_and_state_kept(tiny_w):
+    pb = _pb()
+    w = copy.copy(tiny_w)
+    w["lm_head"] = tiny_w["lm_head"].clone()
+    w["lm_head"][17, 3] = float("nan")
+    ctx = pb.PassContext(TINY, si.weights_to(w, "cuda:0"), 1, 64)
+    ctx.prefill(0, si.make_prompt(TINY, 8))
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(2, 1.0, np.full((1, 5), 0.5, dtype=np.float32))
+    assert e.value.code == -5
+    assert ctx.get_debug(pb.PASS_DBG_KV_LEN)[0] == 7          # unchanged
+    assert ctx.get_debug(pb.PASS_DBG_STATUS)[0] == 0          # cleared for the next call
+    ctx.close()
+
+
+def test_enqueue_collect_matches_step(tiny_w):
+    pb = _pb()
+    prompt = si.make_prompt(TINY, 20)
+    a = pb.PassContext(TINY, si.weights_to(tiny_w, "cuda:0"), 1, 160)
+    b = pb.PassContext(TINY, si.weights_to(tiny_w, "cuda:0"), 1, 160)
+    a.prefill(0, prompt)
+    b.prefill(0, prompt)
+    out_a, out_b = [], []
+    us = [si.step_uniforms(3, 0, s, 5) for s in range(10)]
+    for s in range(10):
+        e, _ = a.step(2, 1.0, us[s].numpy()[None])
+        out_a += e[0]
+    udev = [u.cuda() for u in us]
+    for s in range(10):
+        b.step_enqueue(2, 1.0, udev[s])
+    # only the last step's result is fetched; lengths tell the rest
+    e, _ = b.step_collect()
+    assert a.get_debug(pb.PASS_DBG_KV_LEN)[0] == b.get_debug(pb.PASS_DBG_KV_LEN)[0]
+    assert a.get_debug(pb.PASS_DBG_PENDING)[0] == b.get_debug(pb.PASS_DBG_PENDING)[0]
+    assert out_a[-len(e[0]):] == e[0]
+    assert a.last_step_launches() > 10
+    a.close()
+    b.close()
