@@ -192,6 +192,19 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_HIDDEN        8  /* float32 [rows][d_model]: residual stream after the last layer */
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
+/*
+ * One weight-streaming GEMM of the step on its own (bf16 models only): the "forward pass on n
+ * tokens" reduced to a single matrix, y[r][n] = sum_k x[r][k] W[n][k] for R <= PASS_MAX_ROWS rows.
+ *   which : 0 wq, 1 wk, 2 wv, 3 wo, 4 wg, 5 wu, 6 wd (K = d_ffn), 7 lm_head (layer ignored),
+ *           8 gate|up as the step reads them: output blocks of 128 = 64 gate then 64 up features,
+ *           N = ceil(d_ffn/64)*128.
+ *   x_device [R][K] float32, y_device [R][N] float32, both on the device.  Synchronises.
+ * For tests and for timing the kernel by itself.  Errors: INVALID_ARG, STATE (float32 model),
+ * TIMEOUT, CUDA.
+ */
+int pass_debug_linear(pass_ctx *ctx, int which, int layer, const float *x_device, int R,
+                      float *y_device);
+
 /* Number of kernel launches (graph nodes) of the last pass_step / pass_step_enqueue. */
 int pass_last_step_launches(pass_ctx *ctx);
 /* Stream of the context (a cudaStream_t), so that callers can time on it. */

@@ -23,7 +23,7 @@ PASS_MAX_ROWS = 128
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
-           "pass_stream", "pass_destroy", "pass_strerror"]
+           "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear"]
 
 
 class PassError(RuntimeError):
@@ -75,6 +75,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_set_state.argtypes = [vp, ci, ci, ctypes.c_int32]
     lib.pass_get_debug.argtypes = [vp, ci, vp, ctypes.c_size_t]
     lib.pass_last_step_launches.argtypes = [vp]
+    lib.pass_debug_linear.argtypes = [vp, ci, ci, vp, ci, vp]
     lib.pass_stream.restype = vp
     lib.pass_stream.argtypes = [vp]
     lib.pass_destroy.restype = None
@@ -221,6 +222,15 @@ class PassContext:
             a = np.empty(B, dtype=np.int32)
         _check(self.lib, self.lib.pass_get_debug(self.h, what, a.ctypes.data, a.nbytes))
         return a
+
+    def debug_linear(self, which: int, layer: int, x):
+        """x: CUDA float32 [R][K]; returns CUDA float32 [R][N] (see pass_debug_linear)."""
+        d, f = self.shape.d_model, self.shape.d_ffn
+        N = {4: f, 5: f, 7: self.vocab, 8: ((f + 63) // 64) * 128}.get(which, d)
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.torch.float32
+        y = self.torch.empty((x.shape[0], N), dtype=self.torch.float32, device=self.device)
+        _check(self.lib, self.lib.pass_debug_linear(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
+        return y
 
     def last_step_launches(self) -> int:
         return int(self.lib.pass_last_step_launches(self.h))

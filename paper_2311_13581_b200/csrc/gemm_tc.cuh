@@ -1,0 +1,555 @@
+// Weight-streaming skinny GEMM for the bf16 decoder step on sm_100a.
+//
+//   Y[r][n] = sum_k X[r][k] * W[n][k],   r < R <= 128 token rows, W bf16 [N][K] row-major
+//
+// The step is bound by reading W once from HBM (the paper's premise: "reading the full set of
+// parameters from memory ... forms the primary bottleneck"), so the kernel is built around the
+// weight stream:
+//   * W tiles [128 features x 64 k] (128-byte rows, 128B swizzle) arrive by TMA into a shared-memory
+//     ring; the matching activation tile [npad rows x 64 k] rides in the same stage.
+//   * tcgen05.mma with the WEIGHT tile as operand A (M = 128) and the token rows as operand B
+//     (N = npad, a multiple of 16), fp32 accumulators in TMEM: the token dimension is padded to
+//     16s, not to 64/128.  Activations are carried as bf16 hi + bf16 lo rows (x = hi + lo), which
+//     doubles N at no HBM cost and keeps activation rounding out of the result.
+//   * stream-K: the (tile, k-block) units of one GEMM are cut into equal contiguous ranges, one per
+//     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is.
+//     A tile cut across CTAs is reduced by the LAST CTA to arrive (counter per tile), which sums
+//     the partials in k order - deterministic - and runs the fused epilogue.
+//   * warp roles: warp 0 TMA producer, warp 1 TMEM allocation + MMA issue, warps 2-5 epilogue
+//     (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue of one piece
+//     overlaps the main loop of the next.
+//   * programmatic dependent launch: weight tiles do not depend on the previous kernel, so they are
+//     requested before griddepcontrol.wait; only activation loads and the epilogue wait.
+//   * every mbarrier wait is bounded; on expiry the CTA raises kStatusTimeout, drains its copies,
+//     frees TMEM and returns.
+#pragma once
+#include <cuda.h>
+
+#include "pass_common.cuh"
+
+namespace pass {
+
+constexpr int kTileN = 128;
+constexpr int kBlockK = 64;
+constexpr int kGemmThreads = 192;
+constexpr int kATileBytes = kTileN * kBlockK * 2;       // 16 KB
+constexpr long long kWaitCycles = 400000000LL;          // ~0.2 s at 2 GHz
+
+enum GemmEpilogue { kEpiLogits = 0, kEpiQKV = 1, kEpiResid = 2, kEpiSwiGLU = 3 };
+
+struct GemmParams {
+    int n_tiles, kb_per_tile;
+    int seg_tiles0, seg_tiles1;    // plain mode: tiles of weight map 0 and 1 (the rest is map 2)
+    int interleave;                // 1: tile t = rows [64t, 64t+64) of map 0 (gate) and of map 1 (up)
+    int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
+    int stages;
+    int epi;
+    int n_out;                     // output features in total
+    float* partial_ws;             // [gridDim][2][rh][128] fp32
+    int* tile_counters;            // [n_tiles], zero between launches
+    int* status;
+    // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
+    const float* sumsq_in;
+    int n_parts_in;
+    float inv_d_in, eps;
+    // kEpiLogits
+    float* logits;                 // [R][n_out]
+    // kEpiQKV
+    float* q_out;                  // [R][d]
+    const float2* rope_cs;         // [R][dh/2]
+    const int* row_seq;
+    const int* row_pos;
+    ModelDims md;
+    int layer;
+    __nv_bfloat16* kc;
+    __nv_bfloat16* vc;
+    // kEpiResid
+    float* h;                      // [R][d] residual stream, updated in place
+    const __nv_bfloat16* gain_next;
+    __nv_bfloat16* xn_out;         // [2*rh_out.. rows][d]: hi rows then lo rows
+    int xn_lo_row0;                // first lo row of xn_out / act_out
+    float* sumsq_out;              // [n_tiles][kMaxRows]
+    // kEpiSwiGLU
+    __nv_bfloat16* act_out;        // [rows][f]
+};
+
+// ------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: false when the CTA is giving up (another role timed out, or this wait did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* g_status) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 127u) == 127u) {
+            if (*s_abort) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *s_abort = 1;
+                atomicOr(g_status, kStatusTimeout);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                            uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void griddep_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; i++) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void epi_bar() {            // the 128 epilogue threads only
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile with 128-byte rows, 128B swizzle; 8-row groups are
+// 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;                 // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+    d |= (uint64_t)1 << 46;                 // version
+    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return d;
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = npad.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int npad) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(npad >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------ schedule
+struct Piece {
+    int tile, kb0, kb1;      // k-blocks [kb0, kb1) of the tile
+    int n_pieces, index;     // how many CTAs share the tile, and which of them this is (k order)
+    int slot;                // partial slot of this CTA (0 = its first piece, 1 = a later one)
+};
+
+__device__ __forceinline__ long long unit_start(long long c, long long U, long long G) { return c * U / G; }
+__device__ __forceinline__ int unit_owner(long long x, long long U, long long G) {
+    return (int)(((x + 1) * G - 1) / U);
+}
+
+// The it-th piece of CTA `c`; returns false when the CTA's range is exhausted.
+__device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
+    const long long U = (long long)p.n_tiles * p.kb_per_tile;
+    const long long s = unit_start(c, U, G), e = unit_start(c + 1, U, G);
+    if (s >= e) return false;
+    const int t0 = (int)(s / p.kb_per_tile);
+    const int tile = t0 + it;
+    const long long ts = (long long)tile * p.kb_per_tile;
+    if (ts >= e) return false;
+    const long long a = ts > s ? ts : s;
+    const long long b = (ts + p.kb_per_tile) < e ? (ts + p.kb_per_tile) : e;
+    out.tile = tile;
+    out.kb0 = (int)(a - ts);
+    out.kb1 = (int)(b - ts);
+    const int c_first = unit_owner(ts, U, G), c_last = unit_owner(ts + p.kb_per_tile - 1, U, G);
+    out.n_pieces = c_last - c_first + 1;
+    out.index = c - c_first;
+    out.slot = (a == s) ? 0 : 1;
+    return true;
+}
+
+// ------------------------------------------------------------------------------------ epilogues
+// Thread = one feature of the tile (TMEM lane); v[j] = result for token rows c0 .. c0+7.
+struct EpiCtx {
+    int lane_in_tile;        // 0..127
+    float* s_rstd;           // [kMaxRows]
+    float* s_x;              // [128][9] exchange buffer
+};
+
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[8]) {
+    const int L = ec.lane_in_tile;
+    if (p.epi == kEpiLogits) {
+        const int n = tile * kTileN + L;
+        if (n < p.n_out) {
+#pragma unroll
+            for (int j = 0; j < 8; j++)
+                if (c0 + j < p.R) p.logits[(size_t)(c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
+        }
+    } else if (p.epi == kEpiQKV) {
+        const int d = p.md.d, dh = p.md.dh;
+        const int n = tile * kTileN + L;
+        const int which = n / d, c = n % d, head = c / dh, i = c % dh;
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const int r = c0 + j;
+            const float x = v[j] * (r < p.R ? ec.s_rstd[r] : 0.f);
+            const float other = __shfl_xor_sync(0xffffffffu, x, 1);
+            if (r < p.R) {
+                if (which == 2) {
+                    p.vc[kv_index(p.md, p.layer, p.row_seq[r], head, p.row_pos[r]) + i] = __float2bfloat16_rn(x);
+                } else {
+                    const float2 cs = p.rope_cs[(size_t)r * (dh / 2) + (i >> 1)];
+                    const float y = (i & 1) ? other * cs.y + x * cs.x : x * cs.x - other * cs.y;
+                    if (which == 0) p.q_out[(size_t)r * d + c] = y;
+                    else p.kc[kv_index(p.md, p.layer, p.row_seq[r], head, p.row_pos[r]) + i] = __float2bfloat16_rn(y);
+                }
+            }
+        }
+    } else if (p.epi == kEpiResid) {
+        const int d = p.n_out;
+        const int n = tile * kTileN + L;
+        const float g = n < d ? __bfloat162float(p.gain_next[n]) : 0.f;
+        const int warp_q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
+        float ss[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const int r = c0 + j;
+            float hn = 0.f;
+            if (r < p.R && n < d) {
+                hn = p.h[(size_t)r * d + n] + v[j];
+                p.h[(size_t)r * d + n] = hn;
+                __nv_bfloat16 hi, lo;
+                split_bf16(hn * g, hi, lo);
+                p.xn_out[(size_t)r * d + n] = hi;
+                p.xn_out[(size_t)(p.xn_lo_row0 + r) * d + n] = lo;
+            }
+            ss[j] = warp_sum(hn * hn);
+        }
+        epi_bar();                                  // s_x free
+        if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; j++) ec.s_x[warp_q * 8 + j] = ss[j];
+        }
+        epi_bar();
+        if (L < 8 && c0 + L < p.R)
+            p.sumsq_out[(size_t)tile * kMaxRows + c0 + L] =
+                ec.s_x[L] + ec.s_x[8 + L] + ec.s_x[16 + L] + ec.s_x[24 + L];
+    } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
+        epi_bar();                                  // s_x free
+#pragma unroll
+        for (int j = 0; j < 8; j++) ec.s_x[L * 9 + j] = v[j];
+        epi_bar();
+        if (L < 64) {
+            const int n = tile * 64 + L;
+            if (n < p.n_out) {
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    const int r = c0 + j;
+                    if (r < p.R) {
+                        const float rs = ec.s_rstd[r];
+                        const float g = v[j] * rs, u = ec.s_x[(L + 64) * 9 + j] * rs;
+                        __nv_bfloat16 hi, lo;
+                        split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
+                        p.act_out[(size_t)r * p.n_out + n] = hi;
+                        p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
+          const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
+          const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ int s_issued;
+    __shared__ int s_last;
+    __shared__ int s_epi_fail;
+    __shared__ float s_rstd[kMaxRows];
+    __shared__ float s_x[128 * 9];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const uint32_t stage_bytes = kATileBytes + p.npad * 128;
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_full = smem_u32(&s_bars[0]), bar_empty = bar_full + 8 * 16;
+    const uint32_t bar_accf = bar_full + 8 * 32, bar_acce = bar_accf + 16;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * p.npad) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; s++) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
+        s_abort = 0;
+        s_issued = 0;
+        s_epi_fail = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&s_tmem_base), tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    griddep_launch_dependents();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+            bool waited = false, ok = true;
+            int fill = 0;          // stage fills issued so far
+            int held_kb[16];       // k-blocks whose activation tile is still to be requested
+            Piece pc;
+            auto issue_b = [&](int f, int kb) {
+                const int s = f % S;
+                tma_load_2d(tiles_base + s * stage_bytes + kATileBytes, &map_b, bar_full + 8 * s, kb * kBlockK, 0, pol_x);
+            };
+            // Weights do not depend on the previous kernel: up to S weight tiles are requested before
+            // griddepcontrol.wait; the activation tiles of those stages follow right after it.
+            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                    const int s = fill % S;
+                    if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, p.status)) { ok = false; break; }
+                    mbar_expect_tx(bar_full + 8 * s, stage_bytes);
+                    const uint32_t dst = tiles_base + s * stage_bytes;
+                    const int x = kb * kBlockK;
+                    if (p.interleave) {
+                        tma_load_2d(dst, &map_a0, bar_full + 8 * s, x, pc.tile * 64, pol_w);
+                        tma_load_2d(dst + kATileBytes / 2, &map_a1, bar_full + 8 * s, x, pc.tile * 64, pol_w);
+                    } else {
+                        const CUtensorMap* m = &map_a0;
+                        int tl = pc.tile;
+                        if (tl >= p.seg_tiles0) {
+                            tl -= p.seg_tiles0;
+                            m = &map_a1;
+                            if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = &map_a2; }
+                        }
+                        tma_load_2d(dst, m, bar_full + 8 * s, x, tl * kTileN, pol_w);
+                        tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, x, tl * kTileN + 64, pol_w);
+                    }
+                    if (waited) {
+                        issue_b(fill, kb);
+                    } else {
+                        held_kb[fill] = kb;
+                        if (fill + 1 == S) {
+                            griddep_wait();
+                            waited = true;
+                            for (int f = 0; f <= fill; f++) issue_b(f, held_kb[f]);
+                        }
+                    }
+                    fill++;
+                    *(volatile int*)&s_issued = fill;
+                }
+            }
+            if (!waited) {   // fewer than S fills in all (or giving up): complete what was armed
+                griddep_wait();
+                for (int f = 0; f < fill; f++) issue_b(f, held_kb[f]);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issue
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(p.npad);
+            int fill = 0;
+            bool ok = true;
+            Piece pc;
+            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                const int buf = it & 1;
+                if (!mbar_wait(bar_acce + 8 * buf, ((it >> 1) & 1) ^ 1, &s_abort, p.status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * p.npad;
+                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                    const int s = fill % S;
+                    if (!mbar_wait(bar_full + 8 * s, (fill / S) & 1, &s_abort, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = tiles_base + s * stage_bytes, b_addr = a_addr + kATileBytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+#pragma unroll
+                    for (int kk = 0; kk < kBlockK / 16; kk++)
+                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb > pc.kb0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar_empty + 8 * s);      // frees the stage when these MMAs have read it
+                    fill++;
+                }
+                if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (128 threads)
+        const int wq = warp & 3;                      // TMEM lanes 32*wq .. 32*wq+31
+        EpiCtx ec;
+        ec.lane_in_tile = wq * 32 + lane;
+        ec.s_rstd = s_rstd;
+        ec.s_x = s_x;
+        const int et = (warp - 2) * 32 + lane;        // 0..127
+        griddep_wait();
+        for (int r = et; r < p.R; r += 128) {
+            float rs = 1.f;
+            if (p.sumsq_in) {
+                float ss = 0.f;
+                for (int t = 0; t < p.n_parts_in; t++) ss += p.sumsq_in[(size_t)t * kMaxRows + r];
+                rs = rsqrtf(ss * p.inv_d_in + p.eps);
+            }
+            s_rstd[r] = rs;
+        }
+        epi_bar();
+        const size_t slot_floats = (size_t)p.rh * kTileN;
+        Piece pc;
+        bool ok = true;
+        for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+            const int buf = it & 1;
+            // each thread waits for itself; the outcome is made uniform before any barrier is used
+            if (!mbar_wait(bar_accf + 8 * buf, (it >> 1) & 1, &s_abort, p.status)) *(volatile int*)&s_epi_fail = 1;
+            epi_bar();
+            if (*(volatile int*)&s_epi_fail) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * p.npad;
+            const bool whole = pc.n_pieces == 1;
+            float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
+            for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                float hi[8], lo[8];
+                tmem_ld8(t_addr + c0, hi);
+                tmem_ld8(t_addr + p.rh + c0, lo);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 8; j++) hi[j] += lo[j];
+                if (whole) {
+                    epi_store(p, ec, pc.tile, c0, hi);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; j++) my_slot[(size_t)(c0 + j) * kTileN + ec.lane_in_tile] = hi[j];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+            if (!whole) {
+                // the last CTA to deliver its part of the tile sums all parts in k order
+                __threadfence();
+                epi_bar();
+                if (et == 0) {
+                    const int prev = atomicAdd(p.tile_counters + pc.tile, 1);
+                    s_last = (prev == pc.n_pieces - 1);
+                    if (s_last) p.tile_counters[pc.tile] = 0;
+                }
+                epi_bar();
+                if (s_last) {
+                    __threadfence();
+                    const long long U = (long long)p.n_tiles * p.kb_per_tile;
+                    const long long ts = (long long)pc.tile * p.kb_per_tile;
+                    const int c_first = cta - pc.index;
+                    for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                        float acc[8];
+#pragma unroll
+                        for (int j = 0; j < 8; j++) acc[j] = 0.f;
+                        for (int q = 0; q < pc.n_pieces; q++) {
+                            const int cq = c_first + q;
+                            const long long sq = unit_start(cq, U, G);
+                            const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
+                            const float* src = p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats;
+#pragma unroll
+                            for (int j = 0; j < 8; j++)
+                                acc[j] += __ldcg(src + (size_t)(c0 + j) * kTileN + ec.lane_in_tile);
+                        }
+                        epi_store(p, ec, pc.tile, c0, acc);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (s_abort && threadIdx.x == 0) {
+        // let every copy that was requested land before the shared memory is given back
+        const int issued = *(volatile int*)&s_issued;
+        for (int f = issued - S < 0 ? 0 : issued - S; f < issued; f++) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_full + 8 * (f % S), (f / S) & 1))
+                if (clock64() - t0 > kWaitCycles) break;
+        }
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+}  // namespace pass

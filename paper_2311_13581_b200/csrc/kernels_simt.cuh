@@ -197,11 +197,14 @@ __global__ void k_rope_kv(float* __restrict__ qkv, const float2* __restrict__ cs
 // Attention, one CTA per (head, row): row r attends to cached positions 0 .. pos_r.
 // Each warp walks keys warp, warp+4, ... with an online softmax; warps are merged at the end.
 // ---------------------------------------------------------------------------------------
-template <typename KVT, int DH>
+// q: [R][ldq] float32 (rotated queries).  SPLIT = false: out is float32 [R][d];
+// SPLIT = true: out is bf16 [rows][d] holding hi parts in rows r and lo parts in rows lo_row0 + r.
+template <typename KVT, int DH, bool SPLIT>
 __global__ void __launch_bounds__(128)
-k_attn_simple(const float* __restrict__ qkv, const int* __restrict__ row_seq,
+k_attn_simple(const float* __restrict__ qbuf, int ldq, const int* __restrict__ row_seq,
               const int* __restrict__ row_pos, ModelDims md, int layer,
-              const KVT* __restrict__ kc, const KVT* __restrict__ vc, float* __restrict__ out) {
+              const KVT* __restrict__ kc, const KVT* __restrict__ vc, void* __restrict__ out_,
+              int lo_row0) {
     constexpr int E = DH / 32;
     const int head = blockIdx.x, r = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -210,7 +213,7 @@ k_attn_simple(const float* __restrict__ qkv, const int* __restrict__ row_seq,
     float q[E];
 #pragma unroll
     for (int e = 0; e < E; e++)
-        q[e] = qkv[(size_t)r * 3 * md.d + head * DH + lane * E + e] * scale;
+        q[e] = qbuf[(size_t)r * ldq + head * DH + lane * E + e] * scale;
     const KVT* kb = kc + kv_index(md, layer, seq, head, 0);
     const KVT* vb = vc + kv_index(md, layer, seq, head, 0);
     float mx = -INFINITY, l = 0.f, acc[E];
@@ -242,8 +245,50 @@ k_attn_simple(const float* __restrict__ qkv, const int* __restrict__ row_seq,
         float o = 0.f;
 #pragma unroll
         for (int w = 0; w < 4; w++) o += s_acc[w][c] * __expf(s_m[w] - M);
-        out[(size_t)r * md.d + head * DH + c] = o / L;
+        o /= L;
+        if constexpr (SPLIT) {
+            __nv_bfloat16* out = (__nv_bfloat16*)out_;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(o);
+            out[(size_t)r * md.d + head * DH + c] = hi;
+            out[(size_t)(lo_row0 + r) * md.d + head * DH + c] = __float2bfloat16_rn(o - __bfloat162float(hi));
+        } else {
+            ((float*)out_)[(size_t)r * md.d + head * DH + c] = o;
+        }
     }
+}
+
+// After row assembly on the tensor-core path: the input of the first GEMM and the partial sums of
+// squares that its epilogue turns into the RMSNorm factor.  x = h * g is split into bf16 hi + lo
+// rows; sumsq[t][r] = sum of h^2 over features 128t .. 128t+127.
+__global__ void __launch_bounds__(128)
+k_split_norm_input(const float* __restrict__ h, const __nv_bfloat16* __restrict__ g, int d,
+                   __nv_bfloat16* __restrict__ xn, int lo_row0, float* __restrict__ sumsq) {
+    __shared__ float red[4];
+    const int r = blockIdx.x;
+    for (int t = 0; t < d / 128; t++) {
+        const int n = t * 128 + threadIdx.x;
+        const float v = h[(size_t)r * d + n];
+        const float x = v * __bfloat162float(g[n]);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+        xn[(size_t)r * d + n] = hi;
+        xn[(size_t)(lo_row0 + r) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));
+        const float ss = warp_sum(v * v);
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        if (threadIdx.x == 0) sumsq[(size_t)t * kMaxRows + r] = red[0] + red[1] + red[2] + red[3];
+    }
+}
+
+// Plain split of float32 rows into bf16 hi + lo rows (no gain).
+__global__ void k_split_rows(const float* __restrict__ x, int K, __nv_bfloat16* __restrict__ out, int lo_row0) {
+    const int r = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= K) return;
+    const float v = x[(size_t)r * K + c];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    out[(size_t)r * K + c] = hi;
+    out[(size_t)(lo_row0 + r) * K + c] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
 // F[r][j] = silu(G[r][j]) * U[r][j], GU: [R][2f] (gate | up)

@@ -8,12 +8,15 @@
 #include <new>
 #include <vector>
 
+#include "gemm_tc.cuh"
 #include "kernels_simt.cuh"
 #include "kernels_verify.cuh"
 
 using namespace pass;
 
 namespace {
+
+constexpr int kMaxCtas = 160;      // upper bound of CTAs of one GEMM launch (one per SM)
 
 struct Carve {
     size_t off = 0;
@@ -28,6 +31,7 @@ struct Layout {
     size_t states, params, unif, status, row_seq, row_pos, tok, cs, invfreq;
     size_t h, xn, qkv, attn, gu, act, logits;
     size_t E, chunk, row_sum, row_max, amax_val, amax_idx, q_logits, q_E, q_sum, scratch;
+    size_t xn_bf, attn_bf, act_bf, q_out, sumsq_a, sumsq_b, partial_ws, counters;   // tensor-core path
     size_t total;
 };
 
@@ -42,6 +46,7 @@ bool config_ok(const pass_config* c) {
     if (c->kv_capacity < 1) return false;
     if (c->dtype != PASS_DTYPE_FP32 && c->dtype != PASS_DTYPE_BF16) return false;
     if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+    if (c->dtype == PASS_DTYPE_BF16 && c->d_model % 128) return false;
     return true;
 }
 
@@ -77,6 +82,17 @@ Layout make_layout(const pass_config& c) {
     L.q_E = cv.take(B * 2 * c.k_max * V * 8);
     L.q_sum = cv.take(B * 2 * c.k_max * kVerifySplits * 8);
     L.scratch = cv.take(B * kChunks * 8);
+    L.xn_bf = L.attn_bf = L.act_bf = L.q_out = L.sumsq_a = L.sumsq_b = L.partial_ws = L.counters = 0;
+    if (c.dtype == PASS_DTYPE_BF16) {
+        L.xn_bf = cv.take(2 * R * d * 2);
+        L.attn_bf = cv.take(2 * R * d * 2);
+        L.act_bf = cv.take(2 * R * f * 2);
+        L.q_out = cv.take(R * d * 4);
+        L.sumsq_a = cv.take((d / 128 + 1) * R * 4);
+        L.sumsq_b = cv.take((d / 128 + 1) * R * 4);
+        L.partial_ws = cv.take((size_t)kMaxCtas * 2 * R * kTileN * 4);
+        L.counters = cv.take(4096 * 4);
+    }
     L.total = cv.off;
     return L;
 }
@@ -102,6 +118,17 @@ struct pass_ctx {
     float *d_h, *d_xn, *d_qkv, *d_attn, *d_gu, *d_act, *d_logits;
     VerifyBufs vb;
     double* d_scratch;
+    // tensor-core path (bf16 models)
+    __nv_bfloat16 *d_xn_bf = nullptr, *d_attn_bf = nullptr, *d_act_bf = nullptr;
+    float *d_q_out = nullptr, *d_sumsq_a = nullptr, *d_sumsq_b = nullptr, *d_partial = nullptr;
+    int* d_counters = nullptr;
+    int n_sms = 148;
+    bool use_pdl = true;
+    bool use_tc = false;               // bf16 models run the GEMMs on tcgen05
+    std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
+    CUtensorMap tm_lm;
+    struct BMaps { CUtensorMap xn, attn, act; };
+    std::map<int, BMaps> bmaps;        // by npad
     // weights
     bool weights_loaded = false;
     const void *tok_emb, *la_emb, *lm_head, *final_norm;
@@ -173,6 +200,153 @@ __global__ void k_kv_scatter(const KVT* __restrict__ src, ModelDims md, int laye
     }
 }
 
+// ------------------------------------------------------------------------------- tensor-core path (host)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] row-major; box = 64 columns (128 bytes, 128B swizzle) x box_rows rows.
+static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int npad_for(int R) { return ((2 * R + 15) / 16) * 16; }
+
+static int gemm_stages(int npad) {
+    const int stage = kATileBytes + npad * 128;
+    int s = (112 * 1024 - 1024) / stage;
+    if (s < 4) s = std::min(4, (220 * 1024) / stage);
+    return std::max(2, std::min(16, s));
+}
+
+static const pass_ctx::BMaps* get_bmaps(pass_ctx* c, int npad) {
+    auto it = c->bmaps.find(npad);
+    if (it != c->bmaps.end()) return &it->second;
+    pass_ctx::BMaps bm;
+    if (!make_map(&bm.xn, c->d_xn_bf, 2 * kMaxRows, c->md.d, npad)) return nullptr;
+    if (!make_map(&bm.attn, c->d_attn_bf, 2 * kMaxRows, c->md.d, npad)) return nullptr;
+    if (!make_map(&bm.act, c->d_act_bf, 2 * kMaxRows, c->md.f, npad)) return nullptr;
+    return &(c->bmaps[npad] = bm);
+}
+
+static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, int n_out, int epi) {
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.n_tiles = n_tiles;
+    p.kb_per_tile = (K + kBlockK - 1) / kBlockK;
+    p.seg_tiles0 = p.seg_tiles1 = 1 << 30;
+    p.npad = npad;
+    p.rh = npad / 2;
+    p.R = R;
+    p.stages = gemm_stages(npad);
+    p.epi = epi;
+    p.n_out = n_out;
+    p.partial_ws = c->d_partial;
+    p.tile_counters = c->d_counters;
+    p.status = c->d_status;
+    p.eps = c->md.eps;
+    p.md = c->md;
+    p.xn_lo_row0 = npad / 2;
+    return p;
+}
+
+static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                        const CUtensorMap& b, const GemmParams& p) {
+    const size_t smem = (size_t)p.stages * (kATileBytes + p.npad * 128) + 1024;
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+        cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        smem_set = smem;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    const long long units = (long long)p.n_tiles * p.kb_per_tile;
+    cfg.gridDim = dim3((unsigned)std::min<long long>(c->n_sms, units));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, k_gemm_tc, a0, a1, a2, b, p);
+    c->launches++;
+}
+
+// The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
+// attention, O GEMM (+residual, next norm's input), gate/up GEMM (+SwiGLU), down GEMM (+residual).
+static int enqueue_layers_tc(pass_ctx* c, int R, bool head) {
+    const ModelDims& md = c->md;
+    const int d = md.d, f = md.f, npad = npad_for(R), rh = npad / 2;
+    const pass_ctx::BMaps* bm = get_bmaps(c, npad);
+    if (!bm) return PASS_ERR_CUDA;
+    typedef __nv_bfloat16 bf;
+    LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
+    LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
+    const int dt = d / kTileN;
+    for (int l = 0; l < md.n_layers; l++) {
+        {   // q | k | v
+            GemmParams p = gemm_base(c, R, npad, d, 3 * dt, 3 * d, kEpiQKV);
+            p.seg_tiles0 = p.seg_tiles1 = dt;
+            p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
+            p.q_out = c->d_q_out; p.rope_cs = c->d_cs; p.row_seq = c->d_row_seq; p.row_pos = c->d_row_pos;
+            p.layer = l; p.kc = (bf*)c->kv_k; p.vc = (bf*)c->kv_v;
+            launch_gemm(c, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], bm->xn, p);
+        }
+        if (md.dh == 128)
+            LAUNCH(c, (k_attn_simple<bf, 128, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
+        else
+            LAUNCH(c, (k_attn_simple<bf, 64, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
+        {   // attention output projection + residual; prepares the input of the feed-forward norm
+            GemmParams p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
+            p.h = c->d_h; p.gain_next = (const bf*)c->norm_ffn[l]; p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_b;
+            launch_gemm(c, c->tm_wo[l], c->tm_wo[l], c->tm_wo[l], bm->attn, p);
+        }
+        {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
+            GemmParams p = gemm_base(c, R, npad, d, (f + 63) / 64, f, kEpiSwiGLU);
+            p.interleave = 1;
+            p.sumsq_in = c->d_sumsq_b; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
+            p.act_out = c->d_act_bf;
+            launch_gemm(c, c->tm_wg[l], c->tm_wu[l], c->tm_wu[l], bm->xn, p);
+        }
+        {   // down projection + residual; prepares the input of the next norm
+            GemmParams p = gemm_base(c, R, npad, f, dt, d, kEpiResid);
+            p.h = c->d_h;
+            p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
+            p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_a;
+            launch_gemm(c, c->tm_wd[l], c->tm_wd[l], c->tm_wd[l], bm->act, p);
+        }
+    }
+    if (head) {
+        GemmParams p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
+        p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
+        p.logits = c->d_logits;
+        launch_gemm(c, c->tm_lm, c->tm_lm, c->tm_lm, bm->xn, p);
+    }
+    return PASS_OK;
+}
+
 // ------------------------------------------------------------------------------- forward
 template <typename WT>
 static void enqueue_layers(pass_ctx* c, int R) {
@@ -189,9 +363,9 @@ static void enqueue_layers(pass_ctx* c, int R) {
         LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wv[l], d, d, R, c->d_qkv + 2 * d, 3 * d, 0);
         LAUNCH(c, (k_rope_kv<WT>), R, 256, c->d_qkv, c->d_cs, c->d_row_seq, c->d_row_pos, md, l, (WT*)c->kv_k, (WT*)c->kv_v);
         if (md.dh == 128)
-            LAUNCH(c, (k_attn_simple<WT, 128>), dim3(md.H, R), 128, c->d_qkv, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, c->d_attn);
+            LAUNCH(c, (k_attn_simple<WT, 128, false>), dim3(md.H, R), 128, c->d_qkv, 3 * d, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, (void*)c->d_attn, 0);
         else
-            LAUNCH(c, (k_attn_simple<WT, 64>), dim3(md.H, R), 128, c->d_qkv, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, c->d_attn);
+            LAUNCH(c, (k_attn_simple<WT, 64, false>), dim3(md.H, R), 128, c->d_qkv, 3 * d, c->d_row_seq, c->d_row_pos, md, l, (const WT*)c->kv_k, (const WT*)c->kv_v, (void*)c->d_attn, 0);
         LAUNCH(c, (k_gemm_simt<WT, 16>), (d + gw - 1) / gw, gw * 32, c->d_attn, d, (const WT*)c->wo[l], d, d, R, c->d_h, d, 1);
         LAUNCH(c, (k_rmsnorm<WT>), R, 256, c->d_h, (const WT*)c->norm_ffn[l], d, md.eps, c->d_xn);
         LAUNCH(c, (k_gemm_simt<WT, 16>), (f + gw - 1) / gw, gw * 32, c->d_xn, d, (const WT*)c->wg[l], f, d, R, c->d_gu, 2 * f, 0);
@@ -215,8 +389,12 @@ static void enqueue_step(pass_ctx* c, int k) {
     const int M = 1 + 2 * k, R = md.B * M;
     LAUNCH(c, (k_assemble_step<WT>), R, 256, (const WT*)c->tok_emb, (const WT*)c->la_emb, c->d_states,
            c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos);
-    enqueue_layers<WT>(c, R);
-    enqueue_head<WT>(c, R);
+    if (c->use_tc) {
+        enqueue_layers_tc(c, R, true);
+    } else {
+        enqueue_layers<WT>(c, R);
+        enqueue_head<WT>(c, R);
+    }
     LAUNCH(c, k_verify_stats, dim3(R, kVerifySplits), kVerifyThreads, c->vb, c->d_states, c->d_params, M, md.V, md.k_max);
     LAUNCH(c, k_verify_decide, md.B, 1024, c->vb, c->d_states, c->d_params, c->d_unif, M, md.V, md.k_max, c->d_scratch);
 }
@@ -238,8 +416,13 @@ static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool w
         LAUNCH(c, (k_assemble_tokens<__nv_bfloat16>), n, 256, (const __nv_bfloat16*)c->tok_emb,
                (const __nv_bfloat16*)c->la_emb, c->d_states, c->d_tok, seq, c->md.d, c->md.V, c->d_h,
                c->d_row_seq, c->d_row_pos);
-        enqueue_layers<__nv_bfloat16>(c, n);
-        if (want_logits) enqueue_head<__nv_bfloat16>(c, n);
+        if (c->use_tc) {
+            const int rc = enqueue_layers_tc(c, n, want_logits);
+            if (rc != PASS_OK) return rc;
+        } else {
+            enqueue_layers<__nv_bfloat16>(c, n);
+            if (want_logits) enqueue_head<__nv_bfloat16>(c, n);
+        }
     }
     c->last_rows = n;
     CUDA_TRY(cudaGetLastError());
@@ -310,6 +493,22 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     c->vb.q_sum = (double*)(w + L.q_sum);
     c->vb.status = c->d_status;
     c->d_scratch = (double*)(w + L.scratch);
+    if (cfg->dtype == PASS_DTYPE_BF16) {
+        c->d_xn_bf = (__nv_bfloat16*)(w + L.xn_bf);
+        c->d_attn_bf = (__nv_bfloat16*)(w + L.attn_bf);
+        c->d_act_bf = (__nv_bfloat16*)(w + L.act_bf);
+        c->d_q_out = (float*)(w + L.q_out);
+        c->d_sumsq_a = (float*)(w + L.sumsq_a);
+        c->d_sumsq_b = (float*)(w + L.sumsq_b);
+        c->d_partial = (float*)(w + L.partial_ws);
+        c->d_counters = (int*)(w + L.counters);
+        c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
+        c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+            c->n_sms = std::min(sms, kMaxCtas);
+    }
     c->len_ub.assign(cfg->max_batch, 0);
     c->prefilled.assign(cfg->max_batch, 0);
     c->use_graph = getenv("PASS_NO_GRAPH") == nullptr;
@@ -323,6 +522,8 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
 
     // zero the small state region; rotary frequencies theta^(-2i/d_head) in float64
     if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cfg->dtype == PASS_DTYPE_BF16 &&
+        cudaMemsetAsync(w + L.xn_bf, 0, L.total - L.xn_bf, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     std::vector<double> inv(cfg->d_head / 2);
     for (int i = 0; i < cfg->d_head / 2; i++)
         inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
@@ -352,6 +553,18 @@ int pass_load_weights(pass_ctx* c, const pass_weights* w) {
     c->norm_ffn.assign(w->norm_ffn, w->norm_ffn + nl);
     for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
     c->graphs.clear();
+    if (c->use_tc) {
+        const int d = c->md.d, f = c->md.f;
+        std::vector<CUtensorMap>* tms[] = {&c->tm_wq, &c->tm_wk, &c->tm_wv, &c->tm_wo, &c->tm_wg, &c->tm_wu, &c->tm_wd};
+        const std::vector<const void*>* ws[] = {&c->wq, &c->wk, &c->wv, &c->wo, &c->wg, &c->wu, &c->wd};
+        const int rows[] = {d, d, d, d, f, f, d}, cols[] = {d, d, d, d, d, d, f};
+        for (int i = 0; i < 7; i++) {
+            tms[i]->resize(nl);
+            for (int l = 0; l < nl; l++)
+                if (!make_map(&(*tms[i])[l], (*ws[i])[l], rows[i], cols[i], 64)) return PASS_ERR_CUDA;
+        }
+        if (!make_map(&c->tm_lm, c->lm_head, c->md.V, d, 64)) return PASS_ERR_CUDA;
+    }
     c->weights_loaded = true;
     return PASS_OK;
 }
@@ -621,6 +834,50 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
             return PASS_OK;
         default: return PASS_ERR_INVALID_ARG;
     }
+}
+
+int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, int R, float* y_device) {
+    if (!c || !x_device || !y_device || which < 0 || which > 8 || R < 1 || R > kMaxRows) return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
+    if (which != 7 && (layer < 0 || layer >= c->md.n_layers)) return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    const int d = c->md.d, f = c->md.f, npad = npad_for(R), rh = npad / 2;
+    const pass_ctx::BMaps* bm = get_bmaps(c, npad);
+    if (!bm) return PASS_ERR_CUDA;
+    const int K = which == 6 ? f : d;
+    __nv_bfloat16* xb = which == 6 ? c->d_act_bf : c->d_xn_bf;
+    LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x_device, K, xb, rh);
+    const CUtensorMap* a0 = nullptr;
+    const CUtensorMap* a1 = nullptr;
+    int N = d;
+    switch (which) {
+        case 0: a0 = &c->tm_wq[layer]; break;
+        case 1: a0 = &c->tm_wk[layer]; break;
+        case 2: a0 = &c->tm_wv[layer]; break;
+        case 3: a0 = &c->tm_wo[layer]; break;
+        case 4: a0 = &c->tm_wg[layer]; N = f; break;
+        case 5: a0 = &c->tm_wu[layer]; N = f; break;
+        case 6: a0 = &c->tm_wd[layer]; break;
+        case 7: a0 = &c->tm_lm; N = c->md.V; break;
+        default: a0 = &c->tm_wg[layer]; a1 = &c->tm_wu[layer]; N = ((f + 63) / 64) * 128; break;
+    }
+    const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
+    GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
+    p.interleave = which == 8;
+    p.logits = y_device;
+    launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    int status = 0;
+    CUDA_TRY(cudaMemcpy(&status, c->d_status, 4, cudaMemcpyDeviceToHost));
+    if (status) {
+        CUDA_TRY(cudaMemset(c->d_status, 0, 4));
+        return (status & kStatusTimeout) ? PASS_ERR_TIMEOUT : PASS_ERR_STATE;
+    }
+    return PASS_OK;
 }
 
 int pass_last_step_launches(pass_ctx* c) { return c ? c->last_step_launches : 0; }
