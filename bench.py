@@ -36,6 +36,9 @@ WORKLOADS = {
     "7b-k4-ctx2048-T0.8": dict(shape="7b", k=4, prompt=2048, T=0.8, batch=1),
     "7b-k4-ctx8192-T1.0": dict(shape="7b", k=4, prompt=8192, T=1.0, batch=1),
     "tiny-k2-ctx32": dict(shape="tiny", k=2, prompt=32, T=1.0, batch=1),
+    # depth-reduced 7B (same layer shape, 4 layers): small enough for multi-pass ncu captures
+    "7b-l4-k4-ctx512-greedy": dict(shape="7b", k=4, prompt=512, T=0.0, batch=1, n_layers=4),
+    "7b-k0-ctx512-greedy": dict(shape="7b", k=0, prompt=512, T=0.0, batch=1),
 }
 
 
@@ -169,6 +172,8 @@ def main():
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     shape = si.SHAPES[wl["shape"]]
+    if "n_layers" in wl:
+        shape = dataclasses.replace(shape, n_layers=wl["n_layers"])
     if args.impl == "reference":
         run_reference(args, wl, shape)
         return
