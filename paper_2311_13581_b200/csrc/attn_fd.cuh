@@ -1,0 +1,298 @@
+// Split-K ("flash-decoding") attention for the few causal query rows of one PaSS step over a long
+// contiguous bf16 KV cache.  The paper's premise is that a decoding call re-reads "the past keys
+// and values tensors" once whatever the number of rows: here one CTA streams one slice of one
+// head's keys/values exactly once and serves all M <= 32 rows of the sequence from it.
+//
+//   grid  = (heads, sequences, n_split); 128 threads = 4 warps
+//   K/V   : cp.async, 64-key blocks, 3-stage ring in shared memory, 16-byte chunks XOR-swizzled
+//   math  : mma.sync m16n8k16 bf16 (S = Q K^T, O += P V), fp32 online softmax per warp
+//   split : each slice leaves (O, max, sum) partials; the last slice to finish (counter per
+//           sequence and head) merges them in slice order and writes the bf16 hi/lo rows that
+//           feed the output projection.
+// Row i of a sequence sits at position len + i and may attend to keys 0 .. len + i.
+#pragma once
+#include "pass_common.cuh"
+
+namespace pass {
+
+constexpr int kAttnBK = 64;        // keys per block
+constexpr int kAttnStages = 3;
+constexpr int kAttnMaxSplit = 16;
+
+struct AttnParams {
+    const float* q;                // [rows][ldq] rotated queries, float32
+    int ldq;
+    const int* row_seq;            // [rows]
+    const int* row_pos;            // [rows]
+    ModelDims md;
+    int layer;
+    const __nv_bfloat16* kc;
+    const __nv_bfloat16* vc;
+    int M;                         // rows per sequence (1 + 2k)
+    int n_split;
+    float* part_o;                 // [B][H][n_split][32][DH]
+    float* part_ml;                // [B][H][n_split][32][2]
+    int* counters;                 // [B*H], zero between launches
+    __nv_bfloat16* out;            // [rows][d] hi parts, lo parts lo_row0 rows further down
+    int lo_row0;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int DH, int MT>
+__global__ void __launch_bounds__(128)
+k_attn_fd(const AttnParams p) {
+    extern __shared__ __align__(128) uint8_t smem_attn[];
+    constexpr int CH = DH / 8;                       // 16-byte chunks per key
+    constexpr int TILE_BYTES = kAttnBK * DH * 2;     // one K (or V) block
+    constexpr int KPW = 16 * MT;                     // keys per warp and block
+    __shared__ int s_last;
+
+    const int head = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int mt = warp % MT, part = warp / MT;
+    const int M = p.M, row0 = b * M;
+    const int seq = p.row_seq[row0], len = p.row_pos[row0];
+    const int n_tot = len + M;
+    int chunk = (n_tot + p.n_split - 1) / p.n_split;
+    chunk = ((chunk + kAttnBK - 1) / kAttnBK) * kAttnBK;
+    const int k_begin = split * chunk;
+    const int k_end = min(n_tot, k_begin + chunk);
+    const int nb = k_end > k_begin ? (k_end - k_begin + kAttnBK - 1) / kAttnBK : 0;
+
+    const __nv_bfloat16* kbase = p.kc + kv_index(p.md, p.layer, seq, head, 0);
+    const __nv_bfloat16* vbase = p.vc + kv_index(p.md, p.layer, seq, head, 0);
+    const uint32_t sK = smem_u32(smem_attn), sV = sK + kAttnStages * TILE_BYTES;
+
+    auto load_block = [&](int blk) {
+        const int st = blk % kAttnStages;
+        const int kb = k_begin + blk * kAttnBK;
+        for (int idx = tid; idx < kAttnBK * CH; idx += 128) {
+            const int key = idx / CH, c = idx % CH;
+            const int gk = kb + key;
+            const bool ok = gk < k_end;
+            const size_t off = (size_t)(ok ? gk : 0) * DH + c * 8;
+            const uint32_t d = (uint32_t)((key * CH + (c ^ (key & 7))) * 16);
+            cp_async16(sK + st * TILE_BYTES + d, kbase + off, ok ? 16 : 0);
+            cp_async16(sV + st * TILE_BYTES + d, vbase + off, ok ? 16 : 0);
+        }
+    };
+
+    // query fragments (A operand), scaled by log2(e)/sqrt(d_head) so that exp2 can be used
+    uint32_t qf[DH / 16][4];
+    {
+        const float sc = 1.4426950408889634f * rsqrtf((float)DH);
+        const int i0 = mt * 16 + g, i1 = i0 + 8;
+        const float* q0 = p.q + (size_t)(row0 + i0) * p.ldq + head * DH;
+        const float* q1 = p.q + (size_t)(row0 + i1) * p.ldq + head * DH;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ks++) {
+            const int c = ks * 16 + 2 * t;
+            float2 a = make_float2(0.f, 0.f), bq = a, c2 = a, d2 = a;
+            if (i0 < M) { a = *reinterpret_cast<const float2*>(q0 + c); c2 = *reinterpret_cast<const float2*>(q0 + c + 8); }
+            if (i1 < M) { bq = *reinterpret_cast<const float2*>(q1 + c); d2 = *reinterpret_cast<const float2*>(q1 + c + 8); }
+            qf[ks][0] = pack_bf16(a.x * sc, a.y * sc);
+            qf[ks][1] = pack_bf16(bq.x * sc, bq.y * sc);
+            qf[ks][2] = pack_bf16(c2.x * sc, c2.y * sc);
+            qf[ks][3] = pack_bf16(d2.x * sc, d2.y * sc);
+        }
+    }
+
+    float o[DH / 8][4];
+#pragma unroll
+    for (int n = 0; n < DH / 8; n++) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+#pragma unroll
+    for (int st = 0; st < kAttnStages - 1; st++) {
+        if (st < nb) load_block(st);
+        cp_async_commit();
+    }
+    for (int blk = 0; blk < nb; blk++) {
+        cp_async_wait<kAttnStages - 2>();
+        __syncthreads();
+        if (blk + kAttnStages - 1 < nb) load_block(blk + kAttnStages - 1);
+        cp_async_commit();
+        const int st = blk % kAttnStages;
+        const uint32_t kS = sK + st * TILE_BYTES, vS = sV + st * TILE_BYTES;
+#pragma unroll
+        for (int sub = 0; sub < MT; sub++) {
+            const int key0 = part * KPW + sub * 16;          // within the block
+            const int gkey0 = k_begin + blk * kAttnBK + key0;
+            if (gkey0 >= k_end) continue;
+            float s[2][4];
+#pragma unroll
+            for (int n = 0; n < 2; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+            {
+                const int mi = lane >> 3, rr = lane & 7;
+                const int key = key0 + (mi >> 1) * 8 + rr;
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ks++) {
+                    const int c = 2 * ks + (mi & 1);
+                    uint32_t r[4];
+                    ldsm_x4(kS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
+                    mma_bf16_16816(s[0], qf[ks], r[0], r[1]);
+                    mma_bf16_16816(s[1], qf[ks], r[2], r[3]);
+                }
+            }
+            // causal mask: row i sees key j iff j <= len + i
+            const int i0 = mt * 16 + g, i1 = i0 + 8;
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int n = 0; n < 2; n++)
+#pragma unroll
+                for (int e = 0; e < 2; e++) {
+                    const int j = gkey0 + n * 8 + 2 * t + e;
+                    if (j > len + i0 || j >= k_end) s[n][e] = -INFINITY;
+                    if (j > len + i1 || j >= k_end) s[n][2 + e] = -INFINITY;
+                    mx0 = fmaxf(mx0, s[n][e]);
+                    mx1 = fmaxf(mx1, s[n][2 + e]);
+                }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+            const float c0 = mn0 == -INFINITY ? 1.f : exp2f(m_run[0] - mn0);
+            const float c1 = mn1 == -INFINITY ? 1.f : exp2f(m_run[1] - mn1);
+            const float b0 = mn0 == -INFINITY ? 0.f : mn0, b1 = mn1 == -INFINITY ? 0.f : mn1;
+            m_run[0] = mn0;
+            m_run[1] = mn1;
+            float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < 2; n++)
+#pragma unroll
+                for (int e = 0; e < 2; e++) {
+                    s[n][e] = exp2f(s[n][e] - b0);
+                    s[n][2 + e] = exp2f(s[n][2 + e] - b1);
+                    ps0 += s[n][e];
+                    ps1 += s[n][2 + e];
+                }
+            l_run[0] = l_run[0] * c0 + ps0;
+            l_run[1] = l_run[1] * c1 + ps1;
+#pragma unroll
+            for (int n = 0; n < DH / 8; n++) { o[n][0] *= c0; o[n][1] *= c0; o[n][2] *= c1; o[n][3] *= c1; }
+            uint32_t pa[4];
+            pa[0] = pack_bf16(s[0][0], s[0][1]);
+            pa[1] = pack_bf16(s[0][2], s[0][3]);
+            pa[2] = pack_bf16(s[1][0], s[1][1]);
+            pa[3] = pack_bf16(s[1][2], s[1][3]);
+            {
+                const int mi = lane >> 3, rr = lane & 7;
+                const int key = key0 + (mi & 1) * 8 + rr;
+#pragma unroll
+                for (int np = 0; np < DH / 16; np++) {
+                    const int c = 2 * np + (mi >> 1);
+                    uint32_t r[4];
+                    ldsm_x4_trans(vS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
+                    mma_bf16_16816(o[2 * np], pa, r[0], r[1]);
+                    mma_bf16_16816(o[2 * np + 1], pa, r[2], r[3]);
+                }
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    // merge the warps that share an m-tile; shared memory is reused as [4][16][DH] + stats
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+    float* sm_o = reinterpret_cast<float*>(smem_attn);
+    float* sm_m = sm_o + 4 * 16 * DH;
+    float* sm_l = sm_m + 64;
+#pragma unroll
+    for (int n = 0; n < DH / 8; n++) {
+        *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g) * DH + n * 8 + 2 * t)) = make_float2(o[n][0], o[n][1]);
+        *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g + 8) * DH + n * 8 + 2 * t)) = make_float2(o[n][2], o[n][3]);
+    }
+    if (t == 0) {
+        sm_m[warp * 16 + g] = m_run[0]; sm_m[warp * 16 + g + 8] = m_run[1];
+        sm_l[warp * 16 + g] = l_run[0]; sm_l[warp * 16 + g + 8] = l_run[1];
+    }
+    __syncthreads();
+    constexpr int NP = 4 / MT;                       // warps per m-tile
+    const size_t pbase = ((size_t)(b * p.md.H + head) * p.n_split + split) * 32;
+    for (int idx = tid; idx < MT * 16 * DH; idx += 128) {
+        const int i = idx / DH, dcol = idx % DH;     // i = row within the sequence
+        const int tile = i / 16, rr = i % 16;
+        float mm = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < NP; q++) mm = fmaxf(mm, sm_m[(q * MT + tile) * 16 + rr]);
+        float acc = 0.f, ll = 0.f;
+#pragma unroll
+        for (int q = 0; q < NP; q++) {
+            const int w = q * MT + tile;
+            const float mw = sm_m[w * 16 + rr];
+            const float f = mw == -INFINITY ? 0.f : exp2f(mw - mm);
+            acc += sm_o[(w * 16 + rr) * DH + dcol] * f;
+            ll += sm_l[w * 16 + rr] * f;
+        }
+        if (i < M) {
+            if (p.n_split == 1) {
+                const float v = acc / ll;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+                p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            } else {
+                p.part_o[(pbase + i) * DH + dcol] = acc;
+                if (dcol == 0) { p.part_ml[(pbase + i) * 2] = mm; p.part_ml[(pbase + i) * 2 + 1] = ll; }
+            }
+        }
+    }
+    if (p.n_split == 1) return;
+
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int prev = atomicAdd(p.counters + b * p.md.H + head, 1);
+        s_last = prev == p.n_split - 1;
+        if (s_last) p.counters[b * p.md.H + head] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const size_t hb = (size_t)(b * p.md.H + head) * p.n_split * 32;
+    for (int idx = tid; idx < M * DH; idx += 128) {
+        const int i = idx / DH, dcol = idx % DH;
+        float mm = -INFINITY;
+        for (int sidx = 0; sidx < p.n_split; sidx++) mm = fmaxf(mm, __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2));
+        float acc = 0.f, ll = 0.f;
+        for (int sidx = 0; sidx < p.n_split; sidx++) {
+            const float ms = __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2);
+            const float f = ms == -INFINITY ? 0.f : exp2f(ms - mm);
+            acc += __ldcg(p.part_o + (hb + sidx * 32 + i) * DH + dcol) * f;
+            ll += __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2 + 1) * f;
+        }
+        const float v = acc / ll;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+        p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+}
+
+}  // namespace pass

@@ -74,9 +74,6 @@ struct GemmParams {
 };
 
 // ------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -255,6 +252,16 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int d = p.md.d, dh = p.md.dh;
         const int n = tile * kTileN + L;
         const int which = n / d, c = n % d, head = c / dh, i = c % dh;
+        // everything that is read is fetched before the first store, so that the loads overlap
+        int rs[8], rp[8];
+        float2 cs[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const int r = min(c0 + j, p.R - 1);
+            rs[j] = __ldg(p.row_seq + r);
+            rp[j] = __ldg(p.row_pos + r);
+            cs[j] = __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
+        }
 #pragma unroll
         for (int j = 0; j < 8; j++) {
             const int r = c0 + j;
@@ -262,12 +269,11 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             const float other = __shfl_xor_sync(0xffffffffu, x, 1);
             if (r < p.R) {
                 if (which == 2) {
-                    p.vc[kv_index(p.md, p.layer, p.row_seq[r], head, p.row_pos[r]) + i] = __float2bfloat16_rn(x);
+                    p.vc[kv_index(p.md, p.layer, rs[j], head, rp[j]) + i] = __float2bfloat16_rn(x);
                 } else {
-                    const float2 cs = p.rope_cs[(size_t)r * (dh / 2) + (i >> 1)];
-                    const float y = (i & 1) ? other * cs.y + x * cs.x : x * cs.x - other * cs.y;
+                    const float y = (i & 1) ? other * cs[j].y + x * cs[j].x : x * cs[j].x - other * cs[j].y;
                     if (which == 0) p.q_out[(size_t)r * d + c] = y;
-                    else p.kc[kv_index(p.md, p.layer, p.row_seq[r], head, p.row_pos[r]) + i] = __float2bfloat16_rn(y);
+                    else p.kc[kv_index(p.md, p.layer, rs[j], head, rp[j]) + i] = __float2bfloat16_rn(y);
                 }
             }
         }
@@ -276,13 +282,16 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int n = tile * kTileN + L;
         const float g = n < d ? __bfloat162float(p.gain_next[n]) : 0.f;
         const int warp_q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
-        float ss[8];
+        float ss[8], hv[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++)      // all loads first: they are independent of the stores below
+            hv[j] = (c0 + j < p.R && n < d) ? __ldcg(p.h + (size_t)(c0 + j) * d + n) : 0.f;
 #pragma unroll
         for (int j = 0; j < 8; j++) {
             const int r = c0 + j;
             float hn = 0.f;
             if (r < p.R && n < d) {
-                hn = p.h[(size_t)r * d + n] + v[j];
+                hn = hv[j] + v[j];
                 p.h[(size_t)r * d + n] = hn;
                 __nv_bfloat16 hi, lo;
                 split_bf16(hn * g, hi, lo);

@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "attn_fd.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_simt.cuh"
 #include "kernels_verify.cuh"
@@ -32,6 +33,7 @@ struct Layout {
     size_t h, xn, qkv, attn, gu, act, logits;
     size_t E, chunk, row_sum, row_max, amax_val, amax_idx, q_logits, q_E, q_sum, scratch;
     size_t xn_bf, attn_bf, act_bf, q_out, sumsq_a, sumsq_b, partial_ws, counters;   // tensor-core path
+    size_t attn_po, attn_pml, attn_cnt;
     size_t total;
 };
 
@@ -83,6 +85,7 @@ Layout make_layout(const pass_config& c) {
     L.q_sum = cv.take(B * 2 * c.k_max * kVerifySplits * 8);
     L.scratch = cv.take(B * kChunks * 8);
     L.xn_bf = L.attn_bf = L.act_bf = L.q_out = L.sumsq_a = L.sumsq_b = L.partial_ws = L.counters = 0;
+    L.attn_po = L.attn_pml = L.attn_cnt = 0;
     if (c.dtype == PASS_DTYPE_BF16) {
         L.xn_bf = cv.take(2 * R * d * 2);
         L.attn_bf = cv.take(2 * R * d * 2);
@@ -92,6 +95,10 @@ Layout make_layout(const pass_config& c) {
         L.sumsq_b = cv.take((d / 128 + 1) * R * 4);
         L.partial_ws = cv.take((size_t)kMaxCtas * 2 * R * kTileN * 4);
         L.counters = cv.take(4096 * 4);
+        const size_t slices = 2 * kMaxCtas + B * c.n_heads;     // upper bound of B * heads * n_split
+        L.attn_po = cv.take(slices * 32 * c.d_head * 4);
+        L.attn_pml = cv.take(slices * 32 * 2 * 4);
+        L.attn_cnt = cv.take(B * c.n_heads * 4);
     }
     L.total = cv.off;
     return L;
@@ -122,6 +129,8 @@ struct pass_ctx {
     __nv_bfloat16 *d_xn_bf = nullptr, *d_attn_bf = nullptr, *d_act_bf = nullptr;
     float *d_q_out = nullptr, *d_sumsq_a = nullptr, *d_sumsq_b = nullptr, *d_partial = nullptr;
     int* d_counters = nullptr;
+    float *d_attn_po = nullptr, *d_attn_pml = nullptr;
+    int* d_attn_cnt = nullptr;
     int n_sms = 148;
     bool use_pdl = true;
     bool use_tc = false;               // bf16 models run the GEMMs on tcgen05
@@ -296,7 +305,20 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
 
 // The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
 // attention, O GEMM (+residual, next norm's input), gate/up GEMM (+SwiGLU), down GEMM (+residual).
-static int enqueue_layers_tc(pass_ctx* c, int R, bool head) {
+template <int DH, int MT>
+static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
+    constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
+    static bool set = false;
+    if (!set) {
+        cudaFuncSetAttribute(k_attn_fd<DH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        set = true;
+    }
+    k_attn_fd<DH, MT><<<dim3(c->md.H, n_seq, ap.n_split), 128, smem, c->stream>>>(ap);
+    c->launches++;
+}
+
+// R rows = n_seq sequences x M rows each (M = R when n_seq == 1).
+static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
     const ModelDims& md = c->md;
     const int d = md.d, f = md.f, npad = npad_for(R), rh = npad / 2;
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
@@ -314,10 +336,21 @@ static int enqueue_layers_tc(pass_ctx* c, int R, bool head) {
             p.layer = l; p.kc = (bf*)c->kv_k; p.vc = (bf*)c->kv_v;
             launch_gemm(c, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], bm->xn, p);
         }
-        if (md.dh == 128)
+        const int M = R / n_seq;
+        if (M <= 32) {
+            AttnParams ap;
+            ap.q = c->d_q_out; ap.ldq = d; ap.row_seq = c->d_row_seq; ap.row_pos = c->d_row_pos; ap.md = md;
+            ap.layer = l; ap.kc = (const bf*)c->kv_k; ap.vc = (const bf*)c->kv_v; ap.M = M;
+            ap.n_split = std::max(1, std::min(kAttnMaxSplit, (2 * c->n_sms + md.H * n_seq - 1) / (md.H * n_seq)));
+            ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
+            ap.out = c->d_attn_bf; ap.lo_row0 = rh;
+            if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
+            else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
+        } else if (md.dh == 128) {
             LAUNCH(c, (k_attn_simple<bf, 128, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
-        else
+        } else {
             LAUNCH(c, (k_attn_simple<bf, 64, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
+        }
         {   // attention output projection + residual; prepares the input of the feed-forward norm
             GemmParams p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
             p.h = c->d_h; p.gain_next = (const bf*)c->norm_ffn[l]; p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_b;
@@ -390,7 +423,7 @@ static void enqueue_step(pass_ctx* c, int k) {
     LAUNCH(c, (k_assemble_step<WT>), R, 256, (const WT*)c->tok_emb, (const WT*)c->la_emb, c->d_states,
            c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos);
     if (c->use_tc) {
-        enqueue_layers_tc(c, R, true);
+        enqueue_layers_tc(c, R, md.B, true);
     } else {
         enqueue_layers<WT>(c, R);
         enqueue_head<WT>(c, R);
@@ -417,7 +450,7 @@ static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool w
                (const __nv_bfloat16*)c->la_emb, c->d_states, c->d_tok, seq, c->md.d, c->md.V, c->d_h,
                c->d_row_seq, c->d_row_pos);
         if (c->use_tc) {
-            const int rc = enqueue_layers_tc(c, n, want_logits);
+            const int rc = enqueue_layers_tc(c, n, 1, want_logits);
             if (rc != PASS_OK) return rc;
         } else {
             enqueue_layers<__nv_bfloat16>(c, n);
@@ -502,6 +535,9 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_sumsq_b = (float*)(w + L.sumsq_b);
         c->d_partial = (float*)(w + L.partial_ws);
         c->d_counters = (int*)(w + L.counters);
+        c->d_attn_po = (float*)(w + L.attn_po);
+        c->d_attn_pml = (float*)(w + L.attn_pml);
+        c->d_attn_cnt = (int*)(w + L.attn_cnt);
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         int dev = 0, sms = 0;

@@ -213,3 +213,72 @@ def test_enqueue_collect_matches_step(tiny_w):
     assert a.last_step_launches() > 10
     a.close()
     b.close()
+
+
+# ------------------------------------------------------------------ longer contexts
+@pytest.mark.parametrize("k", [4, 8])
+def test_tiny_bf16_long_prompt_many_key_blocks(k):
+    """1500 cached positions: several 64-key blocks per attention slice, ragged tail."""
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY_BF16, 1501)
+    ctx, oracles, _ = make_pair(TINY_BF16, 1, 1501 + 80, [prompt], seed=1)
+    stats, _ = lockstep(ctx, oracles, k, 0.8, 4, check_A=False)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
+def _load_synthetic_cache(ctx, oracle_backends, shape, n_pos, std=1.0):
+    for b, be in enumerate(oracle_backends):
+        for layer in range(shape.n_layers):
+            k, v = si.make_kv(shape, layer, n_pos, seq=b, std=std)
+            ctx.set_kv(b, layer, 0, k, v)
+            be.k[layer, :n_pos] = k.double().numpy()
+            be.v[layer, :n_pos] = v.double().numpy()
+
+
+SEVENB_2L = dataclasses.replace(si.SHAPES["7b"], n_layers=2)
+THIRTEENB_1L = dataclasses.replace(si.SHAPES["13b"], n_layers=1)
+
+
+@pytest.mark.parametrize("k,T,ctx_len", [(4, 0.0, 512), (4, 0.8, 2048), (8, 0.8, 2048), (1, 0.8, 700), (4, 1.0, 8192)])
+def test_7b_layer_shape_depth2_synthetic_cache(k, T, ctx_len):
+    """Full 7B layer shapes (d 4096, 32 heads, ffn 11008, vocab 32000), two layers, with a seeded
+    synthetic cache standing in for the prompt pass at the paper's context lengths."""
+    import paper_2311_13581_b200 as pb
+    from parity_util import lockstep
+    shape = SEVENB_2L
+    w = si.make_weights(shape, seed=0, device="cuda:0")
+    w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
+    cap = ctx_len + 64
+    ctx = pb.PassContext(shape, w, 1, cap)
+    be = po.TransformerBackend(shape, w_cpu, cap)
+    _load_synthetic_cache(ctx, [be], shape, ctx_len)
+    ctx.set_state(0, ctx_len, 11)
+    orc = po.PassOracle.__new__(po.PassOracle)
+    orc.be, orc.len, orc.pending, orc.drafts = be, ctx_len, 11, []
+    orc.Q_dft, orc.k_prev, orc.T_prev, orc.last_logits = np.zeros((0, shape.vocab)), None, None, None
+    stats, _ = lockstep(ctx, [orc], k, T, 3, check_A=(T == 0.0))
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
+def test_13b_layer_shape_batch4_synthetic_cache():
+    import paper_2311_13581_b200 as pb
+    from parity_util import lockstep
+    shape = THIRTEENB_1L
+    w = si.make_weights(shape, seed=0, device="cuda:0")
+    w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
+    B, ctx_len, cap = 4, 1024, 1100
+    ctx = pb.PassContext(shape, w, B, cap)
+    bes = [po.TransformerBackend(shape, w_cpu, cap) for _ in range(B)]
+    _load_synthetic_cache(ctx, bes, shape, ctx_len)
+    orcs = []
+    for b in range(B):
+        ctx.set_state(b, ctx_len - 3 * b, 5 + b)          # ragged lengths
+        orc = po.PassOracle.__new__(po.PassOracle)
+        orc.be, orc.len, orc.pending, orc.drafts = bes[b], ctx_len - 3 * b, 5 + b, []
+        orc.Q_dft, orc.k_prev, orc.T_prev, orc.last_logits = np.zeros((0, shape.vocab)), None, None, None
+        orcs.append(orc)
+    stats, _ = lockstep(ctx, orcs, 4, 1.0, 3, check_A=False)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
