@@ -190,6 +190,8 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_N_ACCEPTED    6  /* int32 [max_batch]: accepted drafts of the last step */
 #define PASS_DBG_STATUS        7  /* int32 [1]: device status word (0 = fine) */
 #define PASS_DBG_HIDDEN        8  /* float32 [rows][d_model]: residual stream after the last layer */
+#define PASS_DBG_TRACE         9  /* uint64 [launch][160][8]: %globaltimer stamps of the last GEMMs run by
+                                     pass_debug_time_linear when PASS_TRACE is set in the environment */
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
 /*
@@ -204,6 +206,14 @@ int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
  */
 int pass_debug_linear(pass_ctx *ctx, int which, int layer, const float *x_device, int R,
                       float *y_device);
+
+/*
+ * Time that kernel: n_launches launches back to back on the context's stream, cycling over the
+ * layers so that every launch streams different weights from HBM (CUDA events; one untimed pass
+ * over the layers first).  which as above, except 7.  Inputs are whatever the activation buffer
+ * holds.  *ms_total receives the elapsed milliseconds.  Synchronises.
+ */
+int pass_debug_time_linear(pass_ctx *ctx, int which, int R, int n_launches, float *ms_total);
 
 /* Number of kernel launches (graph nodes) of the last pass_step / pass_step_enqueue. */
 int pass_last_step_launches(pass_ctx *ctx);

@@ -23,7 +23,8 @@ PASS_MAX_ROWS = 128
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
-           "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear"]
+           "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
+           "pass_debug_time_linear"]
 
 
 class PassError(RuntimeError):
@@ -76,6 +77,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_get_debug.argtypes = [vp, ci, vp, ctypes.c_size_t]
     lib.pass_last_step_launches.argtypes = [vp]
     lib.pass_debug_linear.argtypes = [vp, ci, ci, vp, ci, vp]
+    lib.pass_debug_time_linear.argtypes = [vp, ci, ci, ci, vp]
     lib.pass_stream.restype = vp
     lib.pass_stream.argtypes = [vp]
     lib.pass_destroy.restype = None
@@ -231,6 +233,12 @@ class PassContext:
         y = self.torch.empty((x.shape[0], N), dtype=self.torch.float32, device=self.device)
         _check(self.lib, self.lib.pass_debug_linear(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
         return y
+
+    def debug_time_linear(self, which: int, R: int, n_launches: int) -> float:
+        """Milliseconds for n_launches back-to-back launches of one GEMM, cycling over layers."""
+        ms = ctypes.c_float(0.0)
+        _check(self.lib, self.lib.pass_debug_time_linear(self.h, which, R, n_launches, ctypes.byref(ms)))
+        return float(ms.value)
 
     def last_step_launches(self) -> int:
         return int(self.lib.pass_last_step_launches(self.h))

@@ -71,6 +71,10 @@ k_attn_fd(const AttnParams p) {
     constexpr int KPW = 16 * MT;                     // keys per warp and block
     __shared__ int s_last;
 
+    // Programmatic dependent launch: let the next kernel (the output projection) become resident and
+    // start streaming its weights now; this kernel's inputs come from the previous one, so wait for it.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int head = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int mt = warp % MT, part = warp / MT;

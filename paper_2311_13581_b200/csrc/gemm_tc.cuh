@@ -15,9 +15,9 @@
 //     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is.
 //     A tile cut across CTAs is reduced by the LAST CTA to arrive (counter per tile), which sums
 //     the partials in k order - deterministic - and runs the fused epilogue.
-//   * warp roles: warp 0 TMA producer, warp 1 TMEM allocation + MMA issue, warps 2-5 epilogue
-//     (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue of one piece
-//     overlaps the main loop of the next.
+//   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 7 L2 prefetch of weights ahead
+//     of the ring, warp 1 TMEM allocation + MMA issue, warps 2-5 epilogue (TMEM -> registers -> fused
+//     epilogue); two accumulator buffers so the epilogue of one piece overlaps the main loop of the next.
 //   * programmatic dependent launch: weight tiles do not depend on the previous kernel, so they are
 //     requested before griddepcontrol.wait; only activation loads and the epilogue wait.
 //   * every mbarrier wait is bounded; on expiry the CTA raises kStatusTimeout, drains its copies,
@@ -31,7 +31,7 @@ namespace pass {
 
 constexpr int kTileN = 128;
 constexpr int kBlockK = 64;
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 256;
 constexpr int kATileBytes = kTileN * kBlockK * 2;       // 16 KB
 constexpr long long kWaitCycles = 400000000LL;          // ~0.2 s at 2 GHz
 
@@ -43,11 +43,13 @@ struct GemmParams {
     int interleave;                // 1: tile t = rows [64t, 64t+64) of map 0 (gate) and of map 1 (up)
     int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
     int stages;
+    int pf_stages;                 // how many stages beyond the ring the producer prefetches into L2
     int epi;
     int n_out;                     // output features in total
     float* partial_ws;             // [gridDim][2][rh][128] fp32
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
+    unsigned long long* trace;     // optional [8 per CTA] timestamps of this launch (nullptr = off)
     // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
     const float* sumsq_in;
     int n_parts_in;
@@ -119,6 +121,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%3, %4}], [%2], %5;"
         ::"r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define PASS_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
+                 ::"l"((uint64_t)map), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
@@ -343,7 +355,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_issued;
+    __shared__ int s_issued, s_issued_b;
     __shared__ int s_last;
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
@@ -360,10 +372,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     while ((int)tmem_cols < 2 * p.npad) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; s++) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        PASS_TRACE(0);
+        for (int s = 0; s < S; s++) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; b++) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
         s_abort = 0;
         s_issued = 0;
+        s_issued_b = 0;
         s_epi_fail = 0;
         fence_barrier_init();
     }
@@ -377,58 +391,102 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     const uint32_t tmem_base = s_tmem_base;
     griddep_launch_dependents();
 
+    // One TMA request costs its issuing thread a couple of hundred cycles, so the requests of a stage
+    // are spread over three single-thread roles in different warps:
+    //   warp 0: weight box 0 of every stage (never waits for the previous kernel: weights are constant)
+    //   warp 6: activation tile of every stage (+ weight box 1 when the stage has two boxes)
+    //   warp 7: runs ahead of the ring and pulls weight tiles into L2
+    // weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box
+    auto weight_box = [&](int tile, int box, const CUtensorMap*& m, int& y) {
+        if (p.interleave) {
+            m = box ? &map_a1 : &map_a0;
+            y = tile * 64;
+        } else {
+            int tl = tile;
+            m = &map_a0;
+            if (tl >= p.seg_tiles0) {
+                tl -= p.seg_tiles0;
+                m = &map_a1;
+                if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = &map_a2; }
+            }
+            y = tl * kTileN;
+        }
+    };
+    const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
     if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
+        // ---------------------------------------------------------------- weight producer
         if (lane == 0) {
-            const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-            bool waited = false, ok = true;
-            int fill = 0;          // stage fills issued so far
-            int held_kb[16];       // k-blocks whose activation tile is still to be requested
+            const uint64_t pol_w = policy_evict_first();
+            int fill = 0;
+            bool ok = true;
             Piece pc;
-            auto issue_b = [&](int f, int kb) {
-                const int s = f % S;
-                tma_load_2d(tiles_base + s * stage_bytes + kATileBytes, &map_b, bar_full + 8 * s, kb * kBlockK, 0, pol_x);
-            };
-            // Weights do not depend on the previous kernel: up to S weight tiles are requested before
-            // griddepcontrol.wait; the activation tiles of those stages follow right after it.
             for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                const CUtensorMap* m;
+                int y;
+                weight_box(pc.tile, 0, m, y);
                 for (int kb = pc.kb0; kb < pc.kb1; kb++) {
                     const int s = fill % S;
                     if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    mbar_expect_tx(bar_full + 8 * s, stage_bytes);
-                    const uint32_t dst = tiles_base + s * stage_bytes;
-                    const int x = kb * kBlockK;
-                    if (p.interleave) {
-                        tma_load_2d(dst, &map_a0, bar_full + 8 * s, x, pc.tile * 64, pol_w);
-                        tma_load_2d(dst + kATileBytes / 2, &map_a1, bar_full + 8 * s, x, pc.tile * 64, pol_w);
-                    } else {
-                        const CUtensorMap* m = &map_a0;
-                        int tl = pc.tile;
-                        if (tl >= p.seg_tiles0) {
-                            tl -= p.seg_tiles0;
-                            m = &map_a1;
-                            if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = &map_a2; }
-                        }
-                        tma_load_2d(dst, m, bar_full + 8 * s, x, tl * kTileN, pol_w);
-                        tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, x, tl * kTileN + 64, pol_w);
-                    }
-                    if (waited) {
-                        issue_b(fill, kb);
-                    } else {
-                        held_kb[fill] = kb;
-                        if (fill + 1 == S) {
-                            griddep_wait();
-                            waited = true;
-                            for (int f = 0; f <= fill; f++) issue_b(f, held_kb[f]);
-                        }
-                    }
+                    mbar_expect_tx(bar_full + 8 * s, a_box_bytes);
+                    tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
                     fill++;
                     *(volatile int*)&s_issued = fill;
                 }
             }
-            if (!waited) {   // fewer than S fills in all (or giving up): complete what was armed
-                griddep_wait();
-                for (int f = 0; f < fill; f++) issue_b(f, held_kb[f]);
+        }
+    } else if (warp == 6) {
+        // ---------------------------------------------------------------- activation producer
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+            int fill = 0;
+            bool ok = true;
+            Piece pc;
+            griddep_wait();                    // activations are the previous kernel's output
+            PASS_TRACE(1);
+            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                const CUtensorMap* m;
+                int y;
+                weight_box(pc.tile, 1, m, y);
+                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                    const int s = fill % S;
+                    if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, p.status)) { ok = false; break; }
+                    const uint32_t dst = tiles_base + s * stage_bytes;
+                    if (p.interleave) {
+                        mbar_expect_tx(bar_full + 8 * s, stage_bytes - a_box_bytes);
+                        tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
+                    } else {
+                        mbar_expect_tx(bar_full + 8 * s, stage_bytes - kATileBytes);
+                    }
+                    tma_load_2d(dst + kATileBytes, &map_b, bar_full + 8 * s, kb * kBlockK, 0, pol_x);
+                    fill++;
+                    *(volatile int*)&s_issued_b = fill;
+                }
+            }
+        }
+    } else if (warp == 7) {
+        // ---------------------------------------------------------------- L2 prefetcher
+        if (lane == 0 && p.pf_stages > 0) {
+            int count = 0;
+            Piece pc;
+            bool stop = false;
+            for (int it = 0; !stop && get_piece(p, cta, G, it, pc); it++) {
+                const CUtensorMap *m0, *m1;
+                int y0, y1;
+                weight_box(pc.tile, 0, m0, y0);
+                weight_box(pc.tile, 1, m1, y1);
+                for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++) {
+                    // stay between the ring and pf_stages beyond it
+                    long long t0 = clock64();
+                    int issued;
+                    while (count >= (issued = *(volatile int*)&s_issued) + S + p.pf_stages) {
+                        if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { stop = true; break; }
+                        __nanosleep(200);
+                    }
+                    if (stop) break;
+                    if (count < issued + S) continue;           // the ring got there first
+                    tma_prefetch_2d(m0, kb * kBlockK, y0);
+                    if (p.interleave) tma_prefetch_2d(m1, kb * kBlockK, y1);
+                }
             }
         }
     } else if (warp == 1) {
@@ -446,6 +504,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                 for (int kb = pc.kb0; kb < pc.kb1; kb++) {
                     const int s = fill % S;
                     if (!mbar_wait(bar_full + 8 * s, (fill / S) & 1, &s_abort, p.status)) { ok = false; break; }
+                    if (fill == 0) PASS_TRACE(2);
                     tc_fence_after();
                     const uint32_t a_addr = tiles_base + s * stage_bytes, b_addr = a_addr + kATileBytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
@@ -457,8 +516,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                 }
                 if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
             }
+            PASS_TRACE(3);
         }
-    } else {
+    } else if (warp >= 2 && warp <= 5) {
         // ---------------------------------------------------------------- epilogue (128 threads)
         const int wq = warp & 3;                      // TMEM lanes 32*wq .. 32*wq+31
         EpiCtx ec;
@@ -486,6 +546,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
             if (!mbar_wait(bar_accf + 8 * buf, (it >> 1) & 1, &s_abort, p.status)) *(volatile int*)&s_epi_fail = 1;
             epi_bar();
             if (*(volatile int*)&s_epi_fail) { ok = false; break; }
+            if (et == 0) PASS_TRACE(4);            // overwritten per piece: the last one stays
             tc_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * p.npad;
             const bool whole = pc.n_pieces == 1;
@@ -500,8 +561,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                 if (whole) {
                     epi_store(p, ec, pc.tile, c0, hi);
                 } else {
-#pragma unroll
-                    for (int j = 0; j < 8; j++) my_slot[(size_t)(c0 + j) * kTileN + ec.lane_in_tile] = hi[j];
+                    // partial slot layout [feature][rh]: each thread owns 4*rh contiguous bytes
+                    float4* dst = reinterpret_cast<float4*>(my_slot + (size_t)ec.lane_in_tile * p.rh + c0);
+                    dst[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    dst[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
                 }
             }
             tc_fence_before();
@@ -526,14 +589,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                         float acc[8];
 #pragma unroll
                         for (int j = 0; j < 8; j++) acc[j] = 0.f;
-                        for (int q = 0; q < pc.n_pieces; q++) {
-                            const int cq = c_first + q;
-                            const long long sq = unit_start(cq, U, G);
-                            const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
-                            const float* src = p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats;
+                        // parts are added in k order; loads go out four parts at a time so that their
+                        // latencies overlap
+                        for (int q0 = 0; q0 < pc.n_pieces; q0 += 4) {
+                            float4 v[4][2];
 #pragma unroll
-                            for (int j = 0; j < 8; j++)
-                                acc[j] += __ldcg(src + (size_t)(c0 + j) * kTileN + ec.lane_in_tile);
+                            for (int qq = 0; qq < 4; qq++) {
+                                const int cq = c_first + min(q0 + qq, pc.n_pieces - 1);
+                                const long long sq = unit_start(cq, U, G);
+                                const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
+                                const float4* src = reinterpret_cast<const float4*>(
+                                    p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * p.rh + c0);
+                                v[qq][0] = __ldcg(src);
+                                v[qq][1] = __ldcg(src + 1);
+                            }
+#pragma unroll
+                            for (int qq = 0; qq < 4; qq++) {
+                                if (q0 + qq < pc.n_pieces) {
+                                    acc[0] += v[qq][0].x; acc[1] += v[qq][0].y; acc[2] += v[qq][0].z; acc[3] += v[qq][0].w;
+                                    acc[4] += v[qq][1].x; acc[5] += v[qq][1].y; acc[6] += v[qq][1].z; acc[7] += v[qq][1].w;
+                                }
+                            }
                         }
                         epi_store(p, ec, pc.tile, c0, acc);
                     }
@@ -543,11 +619,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     }
 
     // ---------------------------------------------------------------- teardown
+    if (threadIdx.x == 64) PASS_TRACE(5);          // first epilogue thread done
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) PASS_TRACE(6);
     if (s_abort && threadIdx.x == 0) {
         // let every copy that was requested land before the shared memory is given back
-        const int issued = *(volatile int*)&s_issued;
+        const int ia = *(volatile int*)&s_issued, ib = *(volatile int*)&s_issued_b;
+        const int issued = ia < ib ? ia : ib;       // stages armed by both producers complete
         for (int f = issued - S < 0 ? 0 : issued - S; f < issued; f++) {
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_full + 8 * (f % S), (f / S) & 1))

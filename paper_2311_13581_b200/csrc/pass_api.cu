@@ -133,8 +133,11 @@ struct pass_ctx {
     int* d_attn_cnt = nullptr;
     int n_sms = 148;
     bool use_pdl = true;
-    bool use_tc = false;               // bf16 models run the GEMMs on tcgen05
+    bool use_tc = false;
+    bool trace = false;                // PASS_TRACE=1: GEMM launches of pass_debug_time_linear leave timestamps
+    int trace_launch = 0;               // bf16 models run the GEMMs on tcgen05
     std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
+    std::vector<CUtensorMap> tm_wg_plain, tm_wu_plain;   // 128-row boxes, for running gate or up alone
     CUtensorMap tm_lm;
     struct BMaps { CUtensorMap xn, attn, act; };
     std::map<int, BMaps> bmaps;        // by npad
@@ -243,6 +246,10 @@ static int npad_for(int R) { return ((2 * R + 15) / 16) * 16; }
 
 static int gemm_stages(int npad) {
     const int stage = kATileBytes + npad * 128;
+    if (const char* e = getenv("PASS_GEMM_STAGES")) {
+        const int s = atoi(e);
+        if (s >= 2 && s <= 16 && (size_t)s * stage + 1024 <= 225 * 1024) return s;
+    }
     int s = (112 * 1024 - 1024) / stage;
     if (s < 4) s = std::min(4, (220 * 1024) / stage);
     return std::max(2, std::min(16, s));
@@ -268,6 +275,8 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     p.rh = npad / 2;
     p.R = R;
     p.stages = gemm_stages(npad);
+    p.pf_stages = 0;
+    if (const char* e = getenv("PASS_GEMM_PF")) p.pf_stages = std::max(0, std::min(256, atoi(e)));
     p.epi = epi;
     p.n_out = n_out;
     p.partial_ws = c->d_partial;
@@ -285,6 +294,9 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
     static size_t smem_set = 0;
     if (smem > smem_set) {
         cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        // all of the SM's L1/shared storage as shared memory: lets the CTA of the next launch become
+        // resident (and start pulling weights) while this launch's CTA is still running
+        cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
         smem_set = smem;
     }
     cudaLaunchConfig_t cfg;
@@ -311,9 +323,21 @@ static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
     static bool set = false;
     if (!set) {
         cudaFuncSetAttribute(k_attn_fd<DH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaFuncSetAttribute(k_attn_fd<DH, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
         set = true;
     }
-    k_attn_fd<DH, MT><<<dim3(c->md.H, n_seq, ap.n_split), 128, smem, c->stream>>>(ap);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->md.H, n_seq, ap.n_split);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT>, ap);
     c->launches++;
 }
 
@@ -341,7 +365,8 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
             AttnParams ap;
             ap.q = c->d_q_out; ap.ldq = d; ap.row_seq = c->d_row_seq; ap.row_pos = c->d_row_pos; ap.md = md;
             ap.layer = l; ap.kc = (const bf*)c->kv_k; ap.vc = (const bf*)c->kv_v; ap.M = M;
-            ap.n_split = std::max(1, std::min(kAttnMaxSplit, (2 * c->n_sms + md.H * n_seq - 1) / (md.H * n_seq)));
+            // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
+            ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
             ap.out = c->d_attn_bf; ap.lo_row0 = rh;
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
@@ -540,6 +565,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_attn_cnt = (int*)(w + L.attn_cnt);
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
+        c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) == cudaSuccess &&
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
@@ -597,9 +623,15 @@ int pass_load_weights(pass_ctx* c, const pass_weights* w) {
         for (int i = 0; i < 7; i++) {
             tms[i]->resize(nl);
             for (int l = 0; l < nl; l++)
-                if (!make_map(&(*tms[i])[l], (*ws[i])[l], rows[i], cols[i], 64)) return PASS_ERR_CUDA;
+                if (!make_map(&(*tms[i])[l], (*ws[i])[l], rows[i], cols[i], (i == 4 || i == 5) ? 64 : 128)) return PASS_ERR_CUDA;
         }
-        if (!make_map(&c->tm_lm, c->lm_head, c->md.V, d, 64)) return PASS_ERR_CUDA;
+        if (!make_map(&c->tm_lm, c->lm_head, c->md.V, d, 128)) return PASS_ERR_CUDA;
+        c->tm_wg_plain.resize(nl);
+        c->tm_wu_plain.resize(nl);
+        for (int l = 0; l < nl; l++) {
+            if (!make_map(&c->tm_wg_plain[l], c->wg[l], f, d, 128)) return PASS_ERR_CUDA;
+            if (!make_map(&c->tm_wu_plain[l], c->wu[l], f, d, 128)) return PASS_ERR_CUDA;
+        }
     }
     c->weights_loaded = true;
     return PASS_OK;
@@ -842,6 +874,12 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         CUDA_TRY(cudaMemcpy(dst, what == PASS_DBG_LOGITS ? c->d_logits : c->d_h, n, cudaMemcpyDeviceToHost));
         return PASS_OK;
     }
+    if (what == PASS_DBG_TRACE) {
+        const size_t n = std::min(bytes, (size_t)64 * kMaxCtas * 8 * 8);
+        CUDA_TRY(cudaMemcpy(dst, c->vb.E, n, cudaMemcpyDeviceToHost));
+        c->trace_launch = 0;
+        return PASS_OK;
+    }
     if (what == PASS_DBG_STATUS) {
         if (!need(4)) return PASS_ERR_CAPACITY;
         CUDA_TRY(cudaMemcpy(dst, c->d_status, 4, cudaMemcpyDeviceToHost));
@@ -872,20 +910,11 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
     }
 }
 
-int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, int R, float* y_device) {
-    if (!c || !x_device || !y_device || which < 0 || which > 8 || R < 1 || R > kMaxRows) return PASS_ERR_INVALID_ARG;
-    if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
-    if (which != 7 && (layer < 0 || layer >= c->md.n_layers)) return PASS_ERR_INVALID_ARG;
-    if (c->pending_collect) {
-        const int rc = pass_step_collect(c, nullptr, nullptr);
-        if (rc != PASS_OK) return rc;
-    }
-    const int d = c->md.d, f = c->md.f, npad = npad_for(R), rh = npad / 2;
+static int enqueue_debug_linear(pass_ctx* c, int which, int layer, int R, float* y_device) {
+    const int d = c->md.d, f = c->md.f, npad = npad_for(R);
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     const int K = which == 6 ? f : d;
-    __nv_bfloat16* xb = which == 6 ? c->d_act_bf : c->d_xn_bf;
-    LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x_device, K, xb, rh);
     const CUtensorMap* a0 = nullptr;
     const CUtensorMap* a1 = nullptr;
     int N = d;
@@ -894,8 +923,8 @@ int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, 
         case 1: a0 = &c->tm_wk[layer]; break;
         case 2: a0 = &c->tm_wv[layer]; break;
         case 3: a0 = &c->tm_wo[layer]; break;
-        case 4: a0 = &c->tm_wg[layer]; N = f; break;
-        case 5: a0 = &c->tm_wu[layer]; N = f; break;
+        case 4: a0 = &c->tm_wg_plain[layer]; N = f; break;
+        case 5: a0 = &c->tm_wu_plain[layer]; N = f; break;
         case 6: a0 = &c->tm_wd[layer]; break;
         case 7: a0 = &c->tm_lm; N = c->md.V; break;
         default: a0 = &c->tm_wg[layer]; a1 = &c->tm_wu[layer]; N = ((f + 63) / 64) * 128; break;
@@ -904,9 +933,13 @@ int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, 
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
     p.logits = y_device;
+    if (c->trace && c->trace_launch < 64)      // the verify scratch (E) doubles as the trace buffer
+        p.trace = (unsigned long long*)c->vb.E + (size_t)(c->trace_launch++) * kMaxCtas * 8;
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
-    CUDA_TRY(cudaGetLastError());
-    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    return PASS_OK;
+}
+
+static int debug_status(pass_ctx* c) {
     int status = 0;
     CUDA_TRY(cudaMemcpy(&status, c->d_status, 4, cudaMemcpyDeviceToHost));
     if (status) {
@@ -914,6 +947,49 @@ int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, 
         return (status & kStatusTimeout) ? PASS_ERR_TIMEOUT : PASS_ERR_STATE;
     }
     return PASS_OK;
+}
+
+int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, int R, float* y_device) {
+    if (!c || !x_device || !y_device || which < 0 || which > 8 || R < 1 || R > kMaxRows) return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
+    if (which != 7 && (layer < 0 || layer >= c->md.n_layers)) return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    const int K = which == 6 ? c->md.f : c->md.d;
+    LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x_device, K, which == 6 ? c->d_act_bf : c->d_xn_bf, npad_for(R) / 2);
+    const int rc = enqueue_debug_linear(c, which, layer, R, y_device);
+    if (rc != PASS_OK) return rc;
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    return debug_status(c);
+}
+
+int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float* ms_total) {
+    if (!c || !ms_total || which < 0 || which > 8 || which == 7 || R < 1 || R > kMaxRows || n_launches < 1)
+        return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
+    const int N = which == 8 ? ((c->md.f + 63) / 64) * 128 : (which == 4 || which == 5 ? c->md.f : c->md.d);
+    if (N > c->md.V) return PASS_ERR_CAPACITY;          // results land in the logits buffer
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    cudaEvent_t e0, e1;
+    CUDA_TRY(cudaEventCreate(&e0));
+    CUDA_TRY(cudaEventCreate(&e1));
+    for (int i = 0; i < std::min(n_launches, c->md.n_layers); i++)        // warm-up pass
+        enqueue_debug_linear(c, which, i % c->md.n_layers, R, c->d_logits);
+    CUDA_TRY(cudaEventRecord(e0, c->stream));
+    for (int i = 0; i < n_launches; i++) enqueue_debug_linear(c, which, i % c->md.n_layers, R, c->d_logits);
+    CUDA_TRY(cudaEventRecord(e1, c->stream));
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    CUDA_TRY(cudaEventElapsedTime(ms_total, e0, e1));
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return debug_status(c);
 }
 
 int pass_last_step_launches(pass_ctx* c) { return c ? c->last_step_launches : 0; }
