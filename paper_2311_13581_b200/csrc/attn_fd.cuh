@@ -241,7 +241,7 @@ k_attn_fd(const AttnParams p) {
     __syncthreads();
     constexpr int NP = 4 / MT;                       // warps per m-tile
     const size_t pbase = ((size_t)(b * p.md.H + head) * p.n_split + split) * 32;
-    for (int idx = tid; idx < MT * 16 * DH; idx += 128) {
+    for (int idx = tid; idx < M * DH; idx += 128) {  // live rows only
         const int i = idx / DH, dcol = idx % DH;     // i = row within the sequence
         const int tile = i / 16, rr = i % 16;
         float mm = -INFINITY;
@@ -256,16 +256,14 @@ k_attn_fd(const AttnParams p) {
             acc += sm_o[(w * 16 + rr) * DH + dcol] * f;
             ll += sm_l[w * 16 + rr] * f;
         }
-        if (i < M) {
-            if (p.n_split == 1) {
-                const float v = acc / ll;
-                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-                p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
-            } else {
-                p.part_o[(pbase + i) * DH + dcol] = acc;
-                if (dcol == 0) { p.part_ml[(pbase + i) * 2] = mm; p.part_ml[(pbase + i) * 2 + 1] = ll; }
-            }
+        if (p.n_split == 1) {
+            const float v = acc / ll;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+            p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        } else {
+            p.part_o[(pbase + i) * DH + dcol] = acc;
+            if (dcol == 0) { p.part_ml[(pbase + i) * 2] = mm; p.part_ml[(pbase + i) * 2 + 1] = ll; }
         }
     }
     if (p.n_split == 1) return;
@@ -280,22 +278,50 @@ k_attn_fd(const AttnParams p) {
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    // The last slice merges all slices.  First the (max, sum) pairs of every slice and row go to
+    // shared memory as ready-made weights, then each output element needs one batch of independent
+    // loads: no load waits for a store.
     const size_t hb = (size_t)(b * p.md.H + head) * p.n_split * 32;
-    for (int idx = tid; idx < M * DH; idx += 128) {
-        const int i = idx / DH, dcol = idx % DH;
+    float* sm_f = reinterpret_cast<float*>(smem_attn);             // [n_split][32] weight of slice s for row i
+    for (int i = tid; i < M; i += 128) {
         float mm = -INFINITY;
         for (int sidx = 0; sidx < p.n_split; sidx++) mm = fmaxf(mm, __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2));
-        float acc = 0.f, ll = 0.f;
+        float ll = 0.f;
         for (int sidx = 0; sidx < p.n_split; sidx++) {
             const float ms = __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2);
             const float f = ms == -INFINITY ? 0.f : exp2f(ms - mm);
-            acc += __ldcg(p.part_o + (hb + sidx * 32 + i) * DH + dcol) * f;
             ll += __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2 + 1) * f;
+            sm_f[sidx * 32 + i] = f;
         }
-        const float v = acc / ll;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-        p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-        p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        const float inv = 1.f / ll;
+        for (int sidx = 0; sidx < p.n_split; sidx++) sm_f[sidx * 32 + i] *= inv;
+    }
+    __syncthreads();
+    constexpr int EB = 4;                                          // elements per thread and batch
+    for (int base = 0; base < M * DH; base += 128 * EB) {
+        float vals[EB][kAttnMaxSplit];
+#pragma unroll
+        for (int e = 0; e < EB; e++) {
+            const int idx = min(base + e * 128 + tid, M * DH - 1);
+            const int i = idx / DH, dcol = idx % DH;
+#pragma unroll
+            for (int sidx = 0; sidx < kAttnMaxSplit; sidx++)
+                vals[e][sidx] = sidx < p.n_split ? __ldcg(p.part_o + (hb + sidx * 32 + i) * DH + dcol) : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < EB; e++) {
+            const int idx = base + e * 128 + tid;
+            if (idx < M * DH) {
+                const int i = idx / DH, dcol = idx % DH;
+                float v = 0.f;
+#pragma unroll
+                for (int sidx = 0; sidx < kAttnMaxSplit; sidx++)
+                    if (sidx < p.n_split) v += vals[e][sidx] * sm_f[sidx * 32 + i];
+                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+                p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            }
+        }
     }
 }
 

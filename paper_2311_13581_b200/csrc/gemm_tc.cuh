@@ -571,17 +571,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
             if (!whole) {
-                // the last CTA to deliver its part of the tile sums all parts in k order
-                __threadfence();
+                // The last CTA to deliver its part of the tile sums all parts in k order.  The barrier
+                // orders every thread's partial stores before thread 0's acq_rel atomic (release is
+                // cumulative), and the loads after the second barrier behind its acquire.
                 epi_bar();
                 if (et == 0) {
-                    const int prev = atomicAdd(p.tile_counters + pc.tile, 1);
+                    int prev;
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                                 : "=r"(prev) : "l"(p.tile_counters + pc.tile) : "memory");
                     s_last = (prev == pc.n_pieces - 1);
                     if (s_last) p.tile_counters[pc.tile] = 0;
                 }
                 epi_bar();
                 if (s_last) {
-                    __threadfence();
                     const long long U = (long long)p.n_tiles * p.kb_per_tile;
                     const long long ts = (long long)pc.tile * p.kb_per_tile;
                     const int c_first = cta - pc.index;
@@ -589,12 +591,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                         float acc[8];
 #pragma unroll
                         for (int j = 0; j < 8; j++) acc[j] = 0.f;
-                        // parts are added in k order; loads go out four parts at a time so that their
+                        // parts are added in k order; loads go out eight parts at a time so that their
                         // latencies overlap
-                        for (int q0 = 0; q0 < pc.n_pieces; q0 += 4) {
-                            float4 v[4][2];
+                        for (int q0 = 0; q0 < pc.n_pieces; q0 += 8) {
+                            float4 v[8][2];
 #pragma unroll
-                            for (int qq = 0; qq < 4; qq++) {
+                            for (int qq = 0; qq < 8; qq++) {
                                 const int cq = c_first + min(q0 + qq, pc.n_pieces - 1);
                                 const long long sq = unit_start(cq, U, G);
                                 const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
@@ -604,7 +606,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
                                 v[qq][1] = __ldcg(src + 1);
                             }
 #pragma unroll
-                            for (int qq = 0; qq < 4; qq++) {
+                            for (int qq = 0; qq < 8; qq++) {
                                 if (q0 + qq < pc.n_pieces) {
                                     acc[0] += v[qq][0].x; acc[1] += v[qq][0].y; acc[2] += v[qq][0].z; acc[3] += v[qq][0].w;
                                     acc[4] += v[qq][1].x; acc[5] += v[qq][1].y; acc[6] += v[qq][1].z; acc[7] += v[qq][1].w;

@@ -203,7 +203,7 @@ k_verify_decide(VerifyBufs vb, SeqState* __restrict__ states, const StepParams* 
                 double* __restrict__ scratch /* [B][kChunks] */) {
     __shared__ double sh_d[64];
     __shared__ int sh_i[4];
-    __shared__ int s_a, s_y;
+    __shared__ int s_a;
     __shared__ int s_arg[2 * kMaxLA + 1];
     const int b = blockIdx.x, tid = threadIdx.x;
     SeqState& st = states[b];
