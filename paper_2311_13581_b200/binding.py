@@ -24,7 +24,7 @@ EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_we
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
-           "pass_debug_time_linear"]
+           "pass_debug_time_linear", "pass_linear_noalloc"]
 
 
 class PassError(RuntimeError):
@@ -78,6 +78,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_last_step_launches.argtypes = [vp]
     lib.pass_debug_linear.argtypes = [vp, ci, ci, vp, ci, vp]
     lib.pass_debug_time_linear.argtypes = [vp, ci, ci, ci, vp]
+    lib.pass_linear_noalloc.argtypes = [vp, ci, ci, vp, ci, vp]
     lib.pass_stream.restype = vp
     lib.pass_stream.argtypes = [vp]
     lib.pass_destroy.restype = None
@@ -232,6 +233,16 @@ class PassContext:
         assert x.is_cuda and x.is_contiguous() and x.dtype == self.torch.float32
         y = self.torch.empty((x.shape[0], N), dtype=self.torch.float32, device=self.device)
         _check(self.lib, self.lib.pass_debug_linear(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
+        return y
+
+    def linear_noalloc(self, which: int, layer: int, x, y):
+        """pass_linear_noalloc: same result as debug_linear, split-K scratch inside the library image.
+
+        For callers that may not allocate device memory: ``y`` (CUDA float32 [R][N]) is passed in
+        rather than created here, and at most 16 rows are accepted."""
+        assert x.is_cuda and x.is_contiguous() and x.dtype == self.torch.float32
+        assert y.is_cuda and y.is_contiguous() and y.dtype == self.torch.float32
+        _check(self.lib, self.lib.pass_linear_noalloc(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
         return y
 
     def debug_time_linear(self, which: int, R: int, n_launches: int) -> float:

@@ -992,6 +992,77 @@ int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float*
     return debug_status(c);
 }
 
+// ------------------------------------------------------------------------------- no-allocation linear
+// Scratch of the split-K GEMM (partial sums of tiles shared by several CTAs + one counter per tile)
+// kept inside the library image instead of in caller-provided memory.  Sized for at most
+// kStaticMaxRows token rows; every GPU that loads the library carries these bytes until exit.
+constexpr int kStaticMaxRows = 16;
+constexpr size_t kStaticPartialBytes = (size_t)kMaxCtas * 2 * kStaticMaxRows * kTileN * sizeof(float);
+constexpr size_t kStaticCounterBytes = 4096 * sizeof(int);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartialBytes + kStaticCounterBytes];
+
+// Device address of g_static_scratch per device ordinal.  In host code the symbol's name is only a
+// handle; the address a kernel can use has to be asked for, with that device current.
+static void* g_static_scratch_addr[64] = {nullptr};
+
+int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device, int R, float* y_device) {
+    if (!c || !x_device || !y_device || which < 0 || which > 8 || R < 1) return PASS_ERR_INVALID_ARG;
+    if (R > kStaticMaxRows) {
+        if (getenv("PASS_LOG"))
+            fprintf(stderr, "[pass] pass_linear_noalloc: %d rows exceed the built-in scratch (max %d rows)\n", R, kStaticMaxRows);
+        return PASS_ERR_CAPACITY;
+    }
+    if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
+    if (which != 7 && (layer < 0 || layer >= c->md.n_layers)) return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return PASS_ERR_INVALID_ARG;
+    if (!g_static_scratch_addr[dev]) {          // first call on this device
+        void* ptr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_scratch_addr[dev] = ptr;
+    }
+    char* scratch = (char*)g_static_scratch_addr[dev];
+    // the tile counters must start at zero; the partial sums are always written before they are read
+    CUDA_TRY(cudaMemsetAsync(scratch + kStaticPartialBytes, 0, kStaticCounterBytes, c->stream));
+
+    const int d = c->md.d, f = c->md.f, npad = npad_for(R);
+    const pass_ctx::BMaps* bm = get_bmaps(c, npad);
+    if (!bm) return PASS_ERR_CUDA;
+    const int K = which == 6 ? f : d;
+    LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x_device, K, which == 6 ? c->d_act_bf : c->d_xn_bf, npad / 2);
+    const CUtensorMap* a0 = nullptr;
+    const CUtensorMap* a1 = nullptr;
+    int N = d;
+    switch (which) {
+        case 0: a0 = &c->tm_wq[layer]; break;
+        case 1: a0 = &c->tm_wk[layer]; break;
+        case 2: a0 = &c->tm_wv[layer]; break;
+        case 3: a0 = &c->tm_wo[layer]; break;
+        case 4: a0 = &c->tm_wg_plain[layer]; N = f; break;
+        case 5: a0 = &c->tm_wu_plain[layer]; N = f; break;
+        case 6: a0 = &c->tm_wd[layer]; break;
+        case 7: a0 = &c->tm_lm; N = c->md.V; break;
+        default: a0 = &c->tm_wg[layer]; a1 = &c->tm_wu[layer]; N = ((f + 63) / 64) * 128; break;
+    }
+    const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
+    if (n_tiles > (int)(kStaticCounterBytes / sizeof(int))) return PASS_ERR_CAPACITY;
+    GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
+    p.trace = nullptr;
+    p.interleave = which == 8;
+    p.logits = y_device;
+    p.partial_ws = (float*)scratch;
+    p.tile_counters = (int*)(scratch + kStaticPartialBytes);
+    launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    return debug_status(c);
+}
+
 int pass_last_step_launches(pass_ctx* c) { return c ? c->last_step_launches : 0; }
 void* pass_stream(pass_ctx* c) { return c ? (void*)c->stream : nullptr; }
 

@@ -1,0 +1,54 @@
+"""pass_linear_noalloc: the GEMM with its split-K scratch built into the library image.
+
+Some users of this library run where the device allocator is out of bounds: the serving
+process gave all free HBM to weights and KV cache at start-up, or sits in a latency-critical
+loop where an allocation may stall or fail.  For them the library offers one GEMM entry point
+whose scratch is a fixed array inside the library.  This test calls it through the C ABI twice
+in a row (the array is shared and keeps the previous call's contents, so the second call is
+the one that shows stale state) and compares with the ordinary entry point.  It is collected
+last on purpose, and builds its own context, so it passes alone as well as after the others.
+"""
+import pytest
+import torch
+
+import synthetic_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+MID = si.ModelShape(2, 512, 4, 128, 1384, 2000, k_max=8, dtype="bf16")
+
+
+def test_noalloc_linear_matches_ordinary_entry_twice_in_a_row():
+    import paper_2311_13581_b200 as pb
+    w = si.make_weights(MID, seed=4)
+    ctx = pb.PassContext(MID, si.weights_to(w, "cuda:0"), 1, 64)
+    g = torch.Generator().manual_seed(11)
+    for which, layer, R in ((6, 1, 9), (3, 0, 16), (8, 1, 5), (7, 0, 12)):
+        K = MID.d_ffn if which == 6 else MID.d_model
+        x1 = torch.randn(R, K, generator=g).cuda()
+        x2 = torch.randn(R, K, generator=g).cuda()
+        ref1 = ctx.debug_linear(which, layer, x1)
+        ref2 = ctx.debug_linear(which, layer, x2)
+        y1, y2 = torch.empty_like(ref1), torch.empty_like(ref1)   # outputs are the caller's, made up front
+        before = torch.cuda.memory_stats()["allocation.all.allocated"]     # allocations made so far
+        got1 = ctx.linear_noalloc(which, layer, x1, y1)
+        got2 = ctx.linear_noalloc(which, layer, x2, y2)  # second call: scratch holds call 1's leftovers
+        # torch's allocator was not asked for anything either
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == before
+        for got, ref in ((got1, ref1), (got2, ref2)):
+            rel = (got.double() - ref.double()).norm(dim=1) / ref.double().norm(dim=1)
+            assert float(rel.max()) < 1e-4
+            assert torch.equal(got, ref)                # same kernel, same summation order
+    ctx.close()
+
+
+def test_noalloc_linear_rejects_more_rows_than_its_scratch_holds():
+    import paper_2311_13581_b200 as pb
+    w = si.make_weights(MID, seed=4)
+    ctx = pb.PassContext(MID, si.weights_to(w, "cuda:0"), 1, 64)
+    x = torch.zeros(17, MID.d_model, device="cuda")
+    y = torch.zeros(17, MID.d_model, device="cuda")
+    with pytest.raises(pb.PassError) as e:
+        ctx.linear_noalloc(3, 0, x, y)
+    assert e.value.code == -2
+    ctx.close()
