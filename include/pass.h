@@ -190,8 +190,9 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_N_ACCEPTED    6  /* int32 [max_batch]: accepted drafts of the last step */
 #define PASS_DBG_STATUS        7  /* int32 [1]: device status word (0 = fine) */
 #define PASS_DBG_HIDDEN        8  /* float32 [rows][d_model]: residual stream after the last layer */
-#define PASS_DBG_TRACE         9  /* uint64 [launch][160][8]: %globaltimer stamps of the last GEMMs run by
-                                     pass_debug_time_linear when PASS_TRACE is set in the environment */
+#define PASS_DBG_TRACE         9  /* uint64 [launch][4 GEMMs][CTAs][8]: %globaltimer stamps of the GEMM-chain
+                                     launches since the last read, when PASS_TRACE is set in the environment:
+                                     activations available, first tile ready, last MMA issued, epilogues done */
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
 /*

@@ -15,9 +15,11 @@
 //     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is.
 //     A tile cut across CTAs is reduced by the LAST CTA to arrive (counter per tile), which sums
 //     the partials in k order - deterministic - and runs the fused epilogue.
-//   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 7 L2 prefetch of weights ahead
-//     of the ring, warp 1 TMEM allocation + MMA issue, warps 2-5 epilogue (TMEM -> registers -> fused
-//     epilogue); two accumulator buffers so the epilogue of one piece overlaps the main loop of the next.
+//   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 1 TMEM allocation + MMA issue,
+//     warps 2-5 epilogue (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue
+//     of one piece overlaps the main loop of the next.
+//   * one launch runs a chain of dependent GEMMs (see k_gemm_tc) so that the weight ring never drains
+//     at a GEMM boundary.
 //   * programmatic dependent launch: weight tiles do not depend on the previous kernel, so they are
 //     requested before griddepcontrol.wait; only activation loads and the epilogue wait.
 //   * every mbarrier wait is bounded; on expiry the CTA raises kStatusTimeout, drains its copies,
@@ -43,13 +45,14 @@ struct GemmParams {
     int interleave;                // 1: tile t = rows [64t, 64t+64) of map 0 (gate) and of map 1 (up)
     int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
     int stages;
-    int pf_stages;                 // how many stages beyond the ring the producer prefetches into L2
     int epi;
     int n_out;                     // output features in total
+    const void* w_base[3];         // the weight matrices behind maps 0..2 (for L2 prefetch), [w_rows][w_ld] bf16
+    int w_rows[3];
+    int w_ld;
     float* partial_ws;             // [gridDim][2][rh][128] fp32
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
-    unsigned long long* trace;     // optional [8 per CTA] timestamps of this launch (nullptr = off)
     // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
     const float* sumsq_in;
     int n_parts_in;
@@ -127,7 +130,6 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-#define PASS_TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 8 + (slot)] = global_ns(); } while (0)
 __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
     asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
                  ::"l"((uint64_t)map), "r"(x), "r"(y) : "memory");
@@ -220,6 +222,8 @@ __device__ __forceinline__ int unit_owner(long long x, long long U, long long G)
 // The it-th piece of CTA `c`; returns false when the CTA's range is exhausted.
 __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
     const long long U = (long long)p.n_tiles * p.kb_per_tile;
+    if (G > U) G = (int)U;            // fewer units than CTAs: only the first U CTAs work on this GEMM
+    if (c >= G) return false;
     const long long s = unit_start(c, U, G), e = unit_start(c + 1, U, G);
     if (s >= e) return false;
     const int t0 = (int)(s / p.kb_per_tile);
@@ -347,10 +351,65 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
 }
 
 // ------------------------------------------------------------------------------------ kernel
+// A launch runs a CHAIN of up to kMaxOps dependent GEMMs (for a decoder layer: output projection ->
+// gate|up -> down -> next layer's QKV).  Inside the chain there is no kernel boundary: the weight
+// producer walks straight from the last tile of one GEMM into the first tile of the next, so the
+// shared-memory ring stays full of weights while the consumers wait for the previous GEMM's epilogues.
+// The wait itself is a counter per GEMM ("tiles whose epilogue is complete"), bumped with release
+// semantics by the CTA that finishes a tile and read with acquire semantics by every CTA's activation
+// producer and epilogue warps before they touch the next GEMM.  All CTAs of the grid are resident
+// (one per SM), the counter only ever waits for work of an EARLIER GEMM, and every wait is bounded.
+constexpr int kMaxOps = 4;
+struct ChainMaps { CUtensorMap m[kMaxOps][4]; };      // per GEMM: weight maps 0..2, activation map
+struct ChainParams {
+    int n_ops;
+    int stages;
+    int npad;                  // row padding, shared by all GEMMs of the chain
+    int pf_units;              // how far beyond the ring weights are pulled into L2 while the ring is stalled
+    int* op_done;              // [kMaxOps] tiles completed per GEMM; zero between launches
+    int* ctas_done;            // CTAs that have left the kernel (the last one clears op_done)
+    int* status;
+    unsigned long long* trace;     // optional %globaltimer stamps [kMaxOps][CTA][8] of this launch (nullptr = off)
+    GemmParams op[kMaxOps];
+};
+#define PASS_TRACE(oi, slot) do { if (cp.trace) cp.trace[((size_t)(oi) * gridDim.x + blockIdx.x) * 8 + (slot)] = global_ns(); } while (0)
+
+__device__ __forceinline__ bool wait_count(const int* counter, int target, volatile int* s_abort, int* g_status) {
+    const long long t0 = clock64();
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if (v >= target) return true;
+        if (*s_abort) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *s_abort = 1;
+            atomicOr(g_status, kStatusTimeout);
+            return false;
+        }
+        __nanosleep(64);
+    }
+}
+
+// weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box
+__device__ __forceinline__ void weight_box(const GemmParams& p, const CUtensorMap* m4, int tile, int box,
+                                           const CUtensorMap*& m, int& y) {
+    if (p.interleave) {
+        m = m4 + (box ? 1 : 0);
+        y = tile * 64;
+    } else {
+        int tl = tile;
+        m = m4;
+        if (tl >= p.seg_tiles0) {
+            tl -= p.seg_tiles0;
+            m = m4 + 1;
+            if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = m4 + 2; }
+        }
+        y = tl * kTileN;
+    }
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
-k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
-          const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
-          const GemmParams p) {
+k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
     __shared__ uint32_t s_tmem_base;
@@ -362,17 +421,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     __shared__ float s_x[128 * 9];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int S = p.stages;
+    const int S = cp.stages;
     const int G = gridDim.x, cta = blockIdx.x;
-    const uint32_t stage_bytes = kATileBytes + p.npad * 128;
+    const uint32_t stage_bytes = kATileBytes + cp.npad * 128;
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_u32(&s_bars[0]), bar_empty = bar_full + 8 * 16;
     const uint32_t bar_accf = bar_full + 8 * 32, bar_acce = bar_accf + 16;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < 2 * p.npad) tmem_cols <<= 1;
+    while ((int)tmem_cols < 2 * cp.npad) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        PASS_TRACE(0);
         for (int s = 0; s < S; s++) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; b++) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
         s_abort = 0;
@@ -392,27 +450,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     griddep_launch_dependents();
 
     // One TMA request costs its issuing thread a couple of hundred cycles, so the requests of a stage
-    // are spread over three single-thread roles in different warps:
-    //   warp 0: weight box 0 of every stage (never waits for the previous kernel: weights are constant)
+    // are spread over two single-thread roles in different warps:
+    //   warp 0: weight box 0 of every stage (never waits for anything but ring space: weights are constant)
     //   warp 6: activation tile of every stage (+ weight box 1 when the stage has two boxes)
-    //   warp 7: runs ahead of the ring and pulls weight tiles into L2
-    // weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box
-    auto weight_box = [&](int tile, int box, const CUtensorMap*& m, int& y) {
-        if (p.interleave) {
-            m = box ? &map_a1 : &map_a0;
-            y = tile * 64;
-        } else {
-            int tl = tile;
-            m = &map_a0;
-            if (tl >= p.seg_tiles0) {
-                tl -= p.seg_tiles0;
-                m = &map_a1;
-                if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = &map_a2; }
-            }
-            y = tl * kTileN;
-        }
-    };
-    const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
     if (warp == 0) {
         // ---------------------------------------------------------------- weight producer
         if (lane == 0) {
@@ -420,17 +460,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
             int fill = 0;
             bool ok = true;
             Piece pc;
-            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
-                const CUtensorMap* m;
-                int y;
-                weight_box(pc.tile, 0, m, y);
-                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                    const int s = fill % S;
-                    if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    mbar_expect_tx(bar_full + 8 * s, a_box_bytes);
-                    tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
-                    fill++;
-                    *(volatile int*)&s_issued = fill;
+            for (int oi = 0; ok && oi < cp.n_ops; oi++) {
+                const GemmParams& p = cp.op[oi];
+                const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
+                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                    const CUtensorMap* m;
+                    int y;
+                    weight_box(p, maps.m[oi], pc.tile, 0, m, y);
+                    for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                        const int s = fill % S;
+                        const uint32_t parity = ((fill / S) & 1) ^ 1;
+                        if (!mbar_wait(bar_empty + 8 * s, parity, &s_abort, cp.status)) { ok = false; break; }
+                        mbar_expect_tx(bar_full + 8 * s, a_box_bytes);
+                        tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
+                        fill++;
+                        *(volatile int*)&s_issued = fill;
+                    }
                 }
             }
         }
@@ -441,82 +486,113 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
             int fill = 0;
             bool ok = true;
             Piece pc;
-            griddep_wait();                    // activations are the previous kernel's output
-            PASS_TRACE(1);
-            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
-                const CUtensorMap* m;
-                int y;
-                weight_box(pc.tile, 1, m, y);
-                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                    const int s = fill % S;
-                    if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    const uint32_t dst = tiles_base + s * stage_bytes;
-                    if (p.interleave) {
-                        mbar_expect_tx(bar_full + 8 * s, stage_bytes - a_box_bytes);
-                        tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
-                    } else {
-                        mbar_expect_tx(bar_full + 8 * s, stage_bytes - kATileBytes);
+            griddep_wait();                    // the first GEMM's activations are the previous kernel's output
+            for (int oi = 0; ok && oi < cp.n_ops; oi++) {
+                const GemmParams& p = cp.op[oi];
+                const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
+                if (oi > 0) {
+                    // activations of this GEMM = results of the previous one, written by other SMs
+                    if (!wait_count(cp.op_done + oi - 1, cp.op[oi - 1].n_tiles, &s_abort, cp.status)) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
+                }
+                PASS_TRACE(oi, 0);
+                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                    const CUtensorMap* m;
+                    int y;
+                    weight_box(p, maps.m[oi], pc.tile, 1, m, y);
+                    for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                        const int s = fill % S;
+                        if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
+                        const uint32_t dst = tiles_base + s * stage_bytes;
+                        if (p.interleave) {
+                            mbar_expect_tx(bar_full + 8 * s, stage_bytes - a_box_bytes);
+                            tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
+                        } else {
+                            mbar_expect_tx(bar_full + 8 * s, stage_bytes - kATileBytes);
+                        }
+                        tma_load_2d(dst + kATileBytes, &maps.m[oi][3], bar_full + 8 * s, kb * kBlockK, 0, pol_x);
+                        fill++;
+                        *(volatile int*)&s_issued_b = fill;
                     }
-                    tma_load_2d(dst + kATileBytes, &map_b, bar_full + 8 * s, kb * kBlockK, 0, pol_x);
-                    fill++;
-                    *(volatile int*)&s_issued_b = fill;
                 }
             }
         }
     } else if (warp == 7) {
-        // ---------------------------------------------------------------- L2 prefetcher
-        if (lane == 0 && p.pf_stages > 0) {
+        // ---------------------------------------------------------------- L2 prefetch (plain loads path)
+        // All 32 lanes walk ahead of the ring (by at most pf_units units) and touch the coming weight
+        // rows with prefetch.global.L2: one 128-byte row segment per lane and instruction.  These go
+        // through the load/store path, not through the TMA queue, so they never sit in front of the
+        // ring's own requests; they keep HBM streaming while the consumers wait for an earlier GEMM.
+        if (cp.pf_units > 0) {
             int count = 0;
             Piece pc;
             bool stop = false;
-            for (int it = 0; !stop && get_piece(p, cta, G, it, pc); it++) {
-                const CUtensorMap *m0, *m1;
-                int y0, y1;
-                weight_box(pc.tile, 0, m0, y0);
-                weight_box(pc.tile, 1, m1, y1);
-                for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++) {
-                    // stay between the ring and pf_stages beyond it
-                    long long t0 = clock64();
-                    int issued;
-                    while (count >= (issued = *(volatile int*)&s_issued) + S + p.pf_stages) {
-                        if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { stop = true; break; }
-                        __nanosleep(200);
+            for (int oi = 0; !stop && oi < cp.n_ops; oi++) {
+                const GemmParams& p = cp.op[oi];
+                for (int it = 0; !stop && get_piece(p, cta, G, it, pc); it++) {
+                    // rows of the tile: plain = 128 rows of one matrix; interleaved = 64 rows of two
+                    const char* base0; const char* base1; int row0, nrows0, nrows1;
+                    if (p.interleave) {
+                        base0 = (const char*)p.w_base[0]; base1 = (const char*)p.w_base[1];
+                        row0 = pc.tile * 64; nrows0 = nrows1 = min(64, p.w_rows[0] - row0);
+                    } else {
+                        int tl = pc.tile, seg = 0;
+                        if (tl >= p.seg_tiles0) { tl -= p.seg_tiles0; seg = 1; if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; seg = 2; } }
+                        base0 = (const char*)p.w_base[seg]; base1 = nullptr;
+                        row0 = tl * kTileN; nrows0 = min(kTileN, p.w_rows[seg] - row0); nrows1 = 0;
                     }
-                    if (stop) break;
-                    if (count < issued + S) continue;           // the ring got there first
-                    tma_prefetch_2d(m0, kb * kBlockK, y0);
-                    if (p.interleave) tma_prefetch_2d(m1, kb * kBlockK, y1);
+                    const size_t ldb = (size_t)p.w_ld * 2;
+                    for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++) {
+                        const long long t0 = clock64();
+                        int issued;
+                        while (count >= (issued = *(volatile int*)&s_issued) + S + cp.pf_units) {
+                            if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { stop = true; break; }
+                            __nanosleep(100);
+                        }
+                        if (stop) break;
+                        if (count < issued + S) continue;                   // the ring got there first
+                        const size_t col = (size_t)kb * kBlockK * 2;
+                        if ((kb + 1) * kBlockK > p.w_ld) continue;          // ragged last k-block: leave it to TMA
+                        for (int r = lane; r < nrows0; r += 32)
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base0 + (size_t)(row0 + r) * ldb + col));
+                        for (int r = lane; r < nrows1; r += 32)
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base1 + (size_t)(row0 + r) * ldb + col));
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issue
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(p.npad);
-            int fill = 0;
+            const uint32_t idesc = instr_desc_bf16(cp.npad);
+            int fill = 0, pidx = 0;
             bool ok = true;
             Piece pc;
-            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
-                const int buf = it & 1;
-                if (!mbar_wait(bar_acce + 8 * buf, ((it >> 1) & 1) ^ 1, &s_abort, p.status)) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * p.npad;
-                for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                    const int s = fill % S;
-                    if (!mbar_wait(bar_full + 8 * s, (fill / S) & 1, &s_abort, p.status)) { ok = false; break; }
-                    if (fill == 0) PASS_TRACE(2);
+            for (int oi = 0; ok && oi < cp.n_ops; oi++) {
+                const GemmParams& p = cp.op[oi];
+                bool first = true;
+                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++, pidx++) {
+                    const int buf = pidx & 1;
+                    if (!mbar_wait(bar_acce + 8 * buf, ((pidx >> 1) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = tiles_base + s * stage_bytes, b_addr = a_addr + kATileBytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
+                    const uint32_t d_tmem = tmem_base + buf * cp.npad;
+                    for (int kb = pc.kb0; kb < pc.kb1; kb++) {
+                        const int s = fill % S;
+                        if (!mbar_wait(bar_full + 8 * s, (fill / S) & 1, &s_abort, cp.status)) { ok = false; break; }
+                        if (first) { PASS_TRACE(oi, 1); first = false; }
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles_base + s * stage_bytes, b_addr = a_addr + kATileBytes;
+                        const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(b_addr);
 #pragma unroll
-                    for (int kk = 0; kk < kBlockK / 16; kk++)
-                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb > pc.kb0 || kk > 0) ? 1u : 0u);
-                    umma_commit(bar_empty + 8 * s);      // frees the stage when these MMAs have read it
-                    fill++;
+                        for (int kk = 0; kk < kBlockK / 16; kk++)
+                            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb > pc.kb0 || kk > 0) ? 1u : 0u);
+                        umma_commit(bar_empty + 8 * s);      // frees the stage when these MMAs have read it
+                        fill++;
+                    }
+                    if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
                 }
-                if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
+                PASS_TRACE(oi, 2);
             }
-            PASS_TRACE(3);
         }
     } else if (warp >= 2 && warp <= 5) {
         // ---------------------------------------------------------------- epilogue (128 threads)
@@ -527,104 +603,127 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
         ec.s_x = s_x;
         const int et = (warp - 2) * 32 + lane;        // 0..127
         griddep_wait();
-        for (int r = et; r < p.R; r += 128) {
-            float rs = 1.f;
-            if (p.sumsq_in) {
-                float ss = 0.f;
-                for (int t = 0; t < p.n_parts_in; t++) ss += p.sumsq_in[(size_t)t * kMaxRows + r];
-                rs = rsqrtf(ss * p.inv_d_in + p.eps);
-            }
-            s_rstd[r] = rs;
-        }
-        epi_bar();
-        const size_t slot_floats = (size_t)p.rh * kTileN;
-        Piece pc;
+        int pidx = 0;
         bool ok = true;
-        for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
-            const int buf = it & 1;
-            // each thread waits for itself; the outcome is made uniform before any barrier is used
-            if (!mbar_wait(bar_accf + 8 * buf, (it >> 1) & 1, &s_abort, p.status)) *(volatile int*)&s_epi_fail = 1;
-            epi_bar();
-            if (*(volatile int*)&s_epi_fail) { ok = false; break; }
-            if (et == 0) PASS_TRACE(4);            // overwritten per piece: the last one stays
-            tc_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * p.npad;
-            const bool whole = pc.n_pieces == 1;
-            float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
-            for (int c0 = 0; c0 < p.rh; c0 += 8) {
-                float hi[8], lo[8];
-                tmem_ld8(t_addr + c0, hi);
-                tmem_ld8(t_addr + p.rh + c0, lo);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 8; j++) hi[j] += lo[j];
-                if (whole) {
-                    epi_store(p, ec, pc.tile, c0, hi);
-                } else {
-                    // partial slot layout [feature][rh]: each thread owns 4*rh contiguous bytes
-                    float4* dst = reinterpret_cast<float4*>(my_slot + (size_t)ec.lane_in_tile * p.rh + c0);
-                    dst[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    dst[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
-                }
+        Piece pc;
+        for (int oi = 0; ok && oi < cp.n_ops; oi++) {
+            const GemmParams& p = cp.op[oi];
+            if (oi > 0) {
+                // one thread waits for the previous GEMM; the outcome is made uniform through the barrier
+                if (et == 0 && !wait_count(cp.op_done + oi - 1, cp.op[oi - 1].n_tiles, &s_abort, cp.status))
+                    *(volatile int*)&s_epi_fail = 1;
+                epi_bar();
+                if (*(volatile int*)&s_epi_fail) { ok = false; break; }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
-            if (!whole) {
-                // The last CTA to deliver its part of the tile sums all parts in k order.  The barrier
-                // orders every thread's partial stores before thread 0's acq_rel atomic (release is
-                // cumulative), and the loads after the second barrier behind its acquire.
-                epi_bar();
-                if (et == 0) {
-                    int prev;
-                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
-                                 : "=r"(prev) : "l"(p.tile_counters + pc.tile) : "memory");
-                    s_last = (prev == pc.n_pieces - 1);
-                    if (s_last) p.tile_counters[pc.tile] = 0;
+            for (int r = et; r < p.R; r += 128) {
+                float rs = 1.f;
+                if (p.sumsq_in) {
+                    float ss = 0.f;
+                    for (int t = 0; t < p.n_parts_in; t++) ss += __ldcg(p.sumsq_in + (size_t)t * kMaxRows + r);
+                    rs = rsqrtf(ss * p.inv_d_in + p.eps);
                 }
+                s_rstd[r] = rs;
+            }
+            epi_bar();
+            const size_t slot_floats = (size_t)p.rh * kTileN;
+            const bool signal = oi + 1 < cp.n_ops;   // a later GEMM of the chain waits for this one's tiles
+            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++, pidx++) {
+                const int buf = pidx & 1;
+                // each thread waits for itself; the outcome is made uniform before any barrier is used
+                if (!mbar_wait(bar_accf + 8 * buf, (pidx >> 1) & 1, &s_abort, cp.status)) *(volatile int*)&s_epi_fail = 1;
                 epi_bar();
-                if (s_last) {
-                    const long long U = (long long)p.n_tiles * p.kb_per_tile;
-                    const long long ts = (long long)pc.tile * p.kb_per_tile;
-                    const int c_first = cta - pc.index;
-                    for (int c0 = 0; c0 < p.rh; c0 += 8) {
-                        float acc[8];
+                if (*(volatile int*)&s_epi_fail) { ok = false; break; }
+                if (et == 0) PASS_TRACE(oi, 4);
+                tc_fence_after();
+                const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
+                const bool whole = pc.n_pieces == 1;
+                float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
+                for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                    float hi[8], lo[8];
+                    tmem_ld8(t_addr + c0, hi);
+                    tmem_ld8(t_addr + p.rh + c0, lo);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 8; j++) acc[j] = 0.f;
-                        // parts are added in k order; loads go out eight parts at a time so that their
-                        // latencies overlap
-                        for (int q0 = 0; q0 < pc.n_pieces; q0 += 8) {
-                            float4 v[8][2];
-#pragma unroll
-                            for (int qq = 0; qq < 8; qq++) {
-                                const int cq = c_first + min(q0 + qq, pc.n_pieces - 1);
-                                const long long sq = unit_start(cq, U, G);
-                                const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
-                                const float4* src = reinterpret_cast<const float4*>(
-                                    p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * p.rh + c0);
-                                v[qq][0] = __ldcg(src);
-                                v[qq][1] = __ldcg(src + 1);
-                            }
-#pragma unroll
-                            for (int qq = 0; qq < 8; qq++) {
-                                if (q0 + qq < pc.n_pieces) {
-                                    acc[0] += v[qq][0].x; acc[1] += v[qq][0].y; acc[2] += v[qq][0].z; acc[3] += v[qq][0].w;
-                                    acc[4] += v[qq][1].x; acc[5] += v[qq][1].y; acc[6] += v[qq][1].z; acc[7] += v[qq][1].w;
-                                }
-                            }
-                        }
-                        epi_store(p, ec, pc.tile, c0, acc);
+                    for (int j = 0; j < 8; j++) hi[j] += lo[j];
+                    if (whole) {
+                        epi_store(p, ec, pc.tile, c0, hi);
+                    } else {
+                        // partial slot layout [feature][rh]: each thread owns 4*rh contiguous bytes
+                        float4* dst = reinterpret_cast<float4*>(my_slot + (size_t)ec.lane_in_tile * p.rh + c0);
+                        dst[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                        dst[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+                bool tile_done = whole;
+                if (!whole) {
+                    // The last CTA to deliver its part of the tile sums all parts in k order.  The barrier
+                    // orders every thread's partial stores before thread 0's acq_rel atomic (release is
+                    // cumulative), and the loads after the second barrier behind its acquire.
+                    epi_bar();
+                    if (et == 0) {
+                        int prev;
+                        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                                     : "=r"(prev) : "l"(p.tile_counters + pc.tile) : "memory");
+                        s_last = (prev == pc.n_pieces - 1);
+                        if (s_last) p.tile_counters[pc.tile] = 0;
+                    }
+                    epi_bar();
+                    if (et == 0) PASS_TRACE(oi, 5);
+                    if (s_last) {
+                        tile_done = true;
+                        const long long U = (long long)p.n_tiles * p.kb_per_tile;
+                        const long long ts = (long long)pc.tile * p.kb_per_tile;
+                        const int Ge = G > U ? (int)U : G;
+                        const int c_first = cta - pc.index;
+                        for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                            float acc[8];
+#pragma unroll
+                            for (int j = 0; j < 8; j++) acc[j] = 0.f;
+                            // parts are added in k order; loads go out eight parts at a time so that their
+                            // latencies overlap
+                            for (int q0 = 0; q0 < pc.n_pieces; q0 += 8) {
+                                float4 v[8][2];
+#pragma unroll
+                                for (int qq = 0; qq < 8; qq++) {
+                                    const int cq = c_first + min(q0 + qq, pc.n_pieces - 1);
+                                    const long long sq = unit_start(cq, U, Ge);
+                                    const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
+                                    const float4* src = reinterpret_cast<const float4*>(
+                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * p.rh + c0);
+                                    v[qq][0] = __ldcg(src);
+                                    v[qq][1] = __ldcg(src + 1);
+                                }
+#pragma unroll
+                                for (int qq = 0; qq < 8; qq++) {
+                                    if (q0 + qq < pc.n_pieces) {
+                                        acc[0] += v[qq][0].x; acc[1] += v[qq][0].y; acc[2] += v[qq][0].z; acc[3] += v[qq][0].w;
+                                        acc[4] += v[qq][1].x; acc[5] += v[qq][1].y; acc[6] += v[qq][1].z; acc[7] += v[qq][1].w;
+                                    }
+                                }
+                            }
+                            epi_store(p, ec, pc.tile, c0, acc);
+                        }
+                    }
+                }
+                if (et == 0 && tile_done && !whole) PASS_TRACE(oi, 6);
+                if (signal && tile_done) {
+                    // every thread's stores of this tile happen-before thread 0's release (barrier + cumulativity)
+                    epi_bar();
+                    if (et == 0)
+                        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cp.op_done + oi) : "memory");
+                    if (et == 0) PASS_TRACE(oi, 7);
+                }
             }
+            if (et == 0) PASS_TRACE(oi, 3);
         }
     }
 
     // ---------------------------------------------------------------- teardown
-    if (threadIdx.x == 64) PASS_TRACE(5);          // first epilogue thread done
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) PASS_TRACE(6);
     if (s_abort && threadIdx.x == 0) {
         // let every copy that was requested land before the shared memory is given back
         const int ia = *(volatile int*)&s_issued, ib = *(volatile int*)&s_issued_b;
@@ -639,6 +738,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CU
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (cp.n_ops > 1 && threadIdx.x == 0) {
+        // the last CTA to leave has seen every CTA pass all of its waits: clear the counters for the next launch
+        int prev;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(cp.ctas_done) : "memory");
+        if (prev == G - 1) {
+            for (int i = 0; i < kMaxOps; i++) cp.op_done[i] = 0;
+            *cp.ctas_done = 0;
+        }
     }
 }
 

@@ -33,7 +33,7 @@ struct Layout {
     size_t h, xn, qkv, attn, gu, act, logits;
     size_t E, chunk, row_sum, row_max, amax_val, amax_idx, q_logits, q_E, q_sum, scratch;
     size_t xn_bf, attn_bf, act_bf, q_out, sumsq_a, sumsq_b, partial_ws, counters;   // tensor-core path
-    size_t attn_po, attn_pml, attn_cnt;
+    size_t attn_po, attn_pml, attn_cnt, chain_flags;
     size_t total;
 };
 
@@ -85,7 +85,7 @@ Layout make_layout(const pass_config& c) {
     L.q_sum = cv.take(B * 2 * c.k_max * kVerifySplits * 8);
     L.scratch = cv.take(B * kChunks * 8);
     L.xn_bf = L.attn_bf = L.act_bf = L.q_out = L.sumsq_a = L.sumsq_b = L.partial_ws = L.counters = 0;
-    L.attn_po = L.attn_pml = L.attn_cnt = 0;
+    L.attn_po = L.attn_pml = L.attn_cnt = L.chain_flags = 0;
     if (c.dtype == PASS_DTYPE_BF16) {
         L.xn_bf = cv.take(2 * R * d * 2);
         L.attn_bf = cv.take(2 * R * d * 2);
@@ -93,12 +93,13 @@ Layout make_layout(const pass_config& c) {
         L.q_out = cv.take(R * d * 4);
         L.sumsq_a = cv.take((d / 128 + 1) * R * 4);
         L.sumsq_b = cv.take((d / 128 + 1) * R * 4);
-        L.partial_ws = cv.take((size_t)kMaxCtas * 2 * R * kTileN * 4);
+        L.partial_ws = cv.take((size_t)kMaxOps * kMaxCtas * 2 * R * kTileN * 4);
         L.counters = cv.take(4096 * 4);
         const size_t slices = 2 * kMaxCtas + B * c.n_heads;     // upper bound of B * heads * n_split
         L.attn_po = cv.take(slices * 32 * c.d_head * 4);
         L.attn_pml = cv.take(slices * 32 * 2 * 4);
         L.attn_cnt = cv.take(B * c.n_heads * 4);
+        L.chain_flags = cv.take(2 * kMaxOps * 4);
     }
     L.total = cv.off;
     return L;
@@ -134,8 +135,9 @@ struct pass_ctx {
     int n_sms = 148;
     bool use_pdl = true;
     bool use_tc = false;
-    bool trace = false;                // PASS_TRACE=1: GEMM launches of pass_debug_time_linear leave timestamps
-    int trace_launch = 0;               // bf16 models run the GEMMs on tcgen05
+    bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
+    int trace_launch = 0;
+    int* d_chain_flags = nullptr;      // [kMaxOps] tiles done per GEMM of a chain, [kMaxOps] = CTAs done               // bf16 models run the GEMMs on tcgen05
     std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
     std::vector<CUtensorMap> tm_wg_plain, tm_wu_plain;   // 128-row boxes, for running gate or up alone
     CUtensorMap tm_lm;
@@ -275,8 +277,6 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     p.rh = npad / 2;
     p.R = R;
     p.stages = gemm_stages(npad);
-    p.pf_stages = 0;
-    if (const char* e = getenv("PASS_GEMM_PF")) p.pf_stages = std::max(0, std::min(256, atoi(e)));
     p.epi = epi;
     p.n_out = n_out;
     p.partial_ws = c->d_partial;
@@ -288,9 +288,43 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     return p;
 }
 
-static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
-                        const CUtensorMap& b, const GemmParams& p) {
-    const size_t smem = (size_t)p.stages * (kATileBytes + p.npad * 128) + 1024;
+// One GEMM of a chain with its four tensor maps (weights 0..2, activations).
+struct ChainOp {
+    GemmParams p;
+    CUtensorMap a0, a1, a2, b;
+};
+
+// Launch up to kMaxOps dependent GEMMs as ONE kernel (see k_gemm_tc).  GEMM j of the chain gets its own
+// partial-sum region and tile counters, because its split tiles may be in flight while GEMM j-1 is
+// still being reduced.
+static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
+    ChainMaps maps;
+    ChainParams cp;
+    memset(&cp, 0, sizeof(cp));
+    cp.n_ops = n_ops;
+    cp.stages = ops[0].p.stages;
+    cp.npad = ops[0].p.npad;
+    cp.pf_units = 0;
+    if (const char* e = getenv("PASS_GEMM_PF")) cp.pf_units = std::max(0, std::min(512, atoi(e)));
+    for (int j = 0; j < n_ops; j++)
+        if (!ops[j].p.w_base[0]) cp.pf_units = 0;      // no raw weight pointers given: nothing to prefetch
+    cp.op_done = c->d_chain_flags;
+    cp.ctas_done = c->d_chain_flags + kMaxOps;
+    cp.status = c->d_status;
+    if (c->trace && c->trace_launch < 48)      // the verify scratch (E) doubles as the trace buffer
+        cp.trace = (unsigned long long*)c->vb.E + (size_t)(c->trace_launch++) * kMaxOps * kMaxCtas * 8;
+    const size_t region = (size_t)kMaxCtas * 2 * kMaxRows * kTileN;      // floats per GEMM of the chain
+    for (int j = 0; j < n_ops; j++) {
+        if (ops[j].p.partial_ws == c->d_partial) {
+            ops[j].p.partial_ws = c->d_partial + (size_t)j * region;
+            ops[j].p.tile_counters = c->d_counters + j * 1024;
+        }
+        cp.op[j] = ops[j].p;
+        maps.m[j][0] = ops[j].a0; maps.m[j][1] = ops[j].a1; maps.m[j][2] = ops[j].a2; maps.m[j][3] = ops[j].b;
+    }
+    for (int j = n_ops; j < kMaxOps; j++)
+        for (int q = 0; q < 4; q++) maps.m[j][q] = ops[0].a0;
+    const size_t smem = (size_t)cp.stages * (kATileBytes + cp.npad * 128) + 1024;
     static size_t smem_set = 0;
     if (smem > smem_set) {
         cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -301,7 +335,9 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
-    const long long units = (long long)p.n_tiles * p.kb_per_tile;
+    long long units = 0;
+    for (int j = 0; j < n_ops; j++) units = std::max(units, (long long)ops[j].p.n_tiles * ops[j].p.kb_per_tile);
+    // a chain needs every CTA resident at once (they wait for one another's tiles): one CTA per SM
     cfg.gridDim = dim3((unsigned)std::min<long long>(c->n_sms, units));
     cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = smem;
@@ -311,8 +347,15 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = c->use_pdl ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, k_gemm_tc, a0, a1, a2, b, p);
+    cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, cp);
     c->launches++;
+}
+
+static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                        const CUtensorMap& b, const GemmParams& p) {
+    ChainOp op;
+    op.p = p; op.a0 = a0; op.a1 = a1; op.a2 = a2; op.b = b;
+    launch_chain(c, &op, 1);
 }
 
 // The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
@@ -351,15 +394,37 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
     LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
     LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
     const int dt = d / kTileN;
+    const bool chained = getenv("PASS_NO_CHAIN") == nullptr;
+    ChainOp chain[kMaxOps];
+    int n_chain = 0;
+    auto flush = [&]() {
+        if (n_chain == 0) return;
+        if (chained) launch_chain(c, chain, n_chain);
+        else for (int j = 0; j < n_chain; j++) launch_chain(c, chain + j, 1);
+        n_chain = 0;
+    };
+    auto add = [&](GemmParams p, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                   const CUtensorMap& b, const void* w0, const void* w1, const void* w2, int rows, int ld) {
+        p.w_base[0] = w0; p.w_base[1] = w1; p.w_base[2] = w2;
+        p.w_rows[0] = p.w_rows[1] = p.w_rows[2] = rows;
+        p.w_ld = ld;
+        chain[n_chain].p = p; chain[n_chain].a0 = a0; chain[n_chain].a1 = a1; chain[n_chain].a2 = a2;
+        chain[n_chain].b = b;
+        n_chain++;
+    };
+    auto qkv = [&](int l) {   // q | k | v
+        GemmParams p = gemm_base(c, R, npad, d, 3 * dt, 3 * d, kEpiQKV);
+        p.seg_tiles0 = p.seg_tiles1 = dt;
+        p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
+        p.q_out = c->d_q_out; p.rope_cs = c->d_cs; p.row_seq = c->d_row_seq; p.row_pos = c->d_row_pos;
+        p.layer = l; p.kc = (bf*)c->kv_k; p.vc = (bf*)c->kv_v;
+        add(p, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], bm->xn, c->wq[l], c->wk[l], c->wv[l], d, d);
+    };
+    // Kernels of a step: QKV_0 | per layer: attention, then ONE launch running
+    // O-projection -> gate|up -> down -> (next layer's QKV, or the output head after the last layer).
+    qkv(0);
+    flush();
     for (int l = 0; l < md.n_layers; l++) {
-        {   // q | k | v
-            GemmParams p = gemm_base(c, R, npad, d, 3 * dt, 3 * d, kEpiQKV);
-            p.seg_tiles0 = p.seg_tiles1 = dt;
-            p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
-            p.q_out = c->d_q_out; p.rope_cs = c->d_cs; p.row_seq = c->d_row_seq; p.row_pos = c->d_row_pos;
-            p.layer = l; p.kc = (bf*)c->kv_k; p.vc = (bf*)c->kv_v;
-            launch_gemm(c, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], bm->xn, p);
-        }
         const int M = R / n_seq;
         if (M <= 32) {
             AttnParams ap;
@@ -379,28 +444,31 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
         {   // attention output projection + residual; prepares the input of the feed-forward norm
             GemmParams p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
             p.h = c->d_h; p.gain_next = (const bf*)c->norm_ffn[l]; p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_b;
-            launch_gemm(c, c->tm_wo[l], c->tm_wo[l], c->tm_wo[l], bm->attn, p);
+            add(p, c->tm_wo[l], c->tm_wo[l], c->tm_wo[l], bm->attn, c->wo[l], c->wo[l], c->wo[l], d, d);
         }
         {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
             GemmParams p = gemm_base(c, R, npad, d, (f + 63) / 64, f, kEpiSwiGLU);
             p.interleave = 1;
             p.sumsq_in = c->d_sumsq_b; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
             p.act_out = c->d_act_bf;
-            launch_gemm(c, c->tm_wg[l], c->tm_wu[l], c->tm_wu[l], bm->xn, p);
+            add(p, c->tm_wg[l], c->tm_wu[l], c->tm_wu[l], bm->xn, c->wg[l], c->wu[l], c->wu[l], f, d);
         }
         {   // down projection + residual; prepares the input of the next norm
             GemmParams p = gemm_base(c, R, npad, f, dt, d, kEpiResid);
             p.h = c->d_h;
             p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
             p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_a;
-            launch_gemm(c, c->tm_wd[l], c->tm_wd[l], c->tm_wd[l], bm->act, p);
+            add(p, c->tm_wd[l], c->tm_wd[l], c->tm_wd[l], bm->act, c->wd[l], c->wd[l], c->wd[l], d, f);
         }
-    }
-    if (head) {
-        GemmParams p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
-        p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
-        p.logits = c->d_logits;
-        launch_gemm(c, c->tm_lm, c->tm_lm, c->tm_lm, bm->xn, p);
+        if (l + 1 < md.n_layers) {
+            qkv(l + 1);
+        } else if (head) {
+            GemmParams p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
+            p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
+            p.logits = c->d_logits;
+            add(p, c->tm_lm, c->tm_lm, c->tm_lm, bm->xn, c->lm_head, c->lm_head, c->lm_head, md.V, d);
+        }
+        flush();
     }
     return PASS_OK;
 }
@@ -563,6 +631,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_attn_po = (float*)(w + L.attn_po);
         c->d_attn_pml = (float*)(w + L.attn_pml);
         c->d_attn_cnt = (int*)(w + L.attn_cnt);
+        c->d_chain_flags = (int*)(w + L.chain_flags);
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         c->trace = getenv("PASS_TRACE") != nullptr;
@@ -875,7 +944,7 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         return PASS_OK;
     }
     if (what == PASS_DBG_TRACE) {
-        const size_t n = std::min(bytes, (size_t)64 * kMaxCtas * 8 * 8);
+        const size_t n = std::min(bytes, (size_t)48 * kMaxOps * kMaxCtas * 8 * 8);
         CUDA_TRY(cudaMemcpy(dst, c->vb.E, n, cudaMemcpyDeviceToHost));
         c->trace_launch = 0;
         return PASS_OK;
@@ -933,8 +1002,6 @@ static int enqueue_debug_linear(pass_ctx* c, int which, int layer, int R, float*
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
     p.logits = y_device;
-    if (c->trace && c->trace_launch < 64)      // the verify scratch (E) doubles as the trace buffer
-        p.trace = (unsigned long long*)c->vb.E + (size_t)(c->trace_launch++) * kMaxCtas * 8;
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
     return PASS_OK;
 }
@@ -1052,7 +1119,6 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
     if (n_tiles > (int)(kStaticCounterBytes / sizeof(int))) return PASS_ERR_CAPACITY;
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
-    p.trace = nullptr;
     p.interleave = which == 8;
     p.logits = y_device;
     p.partial_ws = (float*)scratch;
