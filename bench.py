@@ -28,6 +28,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 import synthetic_inputs as si  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_gemm_tc layer-chain launch (7B layer shape, 9 rows),
+# from the ncu capture summarised in profiles/; None whenever the kernel has changed since that capture.
+CHAIN_TRAFFIC_BYTES = None
+
 METRIC = "PaSS ms/step and accepted tok/s at 7B-shape bf16 batch 1; HBM GB/s vs 8 TB/s"
 
 WORKLOADS = {
@@ -242,6 +246,14 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- the dominant kernel by itself: the GEMM chain of one layer (O-proj -> gate|up -> down -> next QKV),
+    # 64 launches back to back cycling over the layers (every launch streams other weights), CUDA events on
+    # the library's stream.  Last, because it scribbles over the residual stream and one cache row.
+    chain_us = None
+    if shape.dtype == "bf16" and shape.n_layers >= 2:
+        n_chain = 64
+        chain_us = min(ctx.debug_time_linear(9, B * (1 + 2 * k), n_chain) for _ in range(3)) * 1e3 / n_chain
+
     t = torch.tensor([ms_total, e2e_s * 1e3, float(tokens), float(tok_e2e)], dtype=torch.float64, device=dev)
     if world > 1:
         tmax = t.clone()
@@ -276,11 +288,21 @@ def main():
         "e2e": {"value": tok_e2e / (e2e_ms * 1e-3), "unit": "tok/s", "ms_per_step": e2e_ms / args.steps,
                 "h2d_bytes_per_step": (B * n_u * 4 if T > 0 else 0),
                 "d2h_bytes_per_step": B * 26 * 4 + 4},
-        "roofline": {"bound": "hbm", "kernel": "pass_step graph (weights + KV stream)",
-                     "achieved": gbs, "peak": pk["hbm_gbs"], "peak_kind": pk_kind, "unit": "GB/s",
-                     "frac": gbs / pk["hbm_gbs"], "traffic": None,
-                     "algorithmic_bytes": bytes_step},
+        "step_roofline": {"bound": "hbm", "what": "whole step: weights + cached K/V read once",
+                          "achieved": gbs, "peak": pk["hbm_gbs"], "peak_kind": pk_kind, "unit": "GB/s",
+                          "frac": gbs / pk["hbm_gbs"], "algorithmic_bytes": bytes_step},
     }
+    if chain_us is not None:
+        es = 2
+        chain_bytes = (4 * shape.d_model * shape.d_model + 3 * shape.d_model * shape.d_ffn) * es
+        ach = chain_bytes / (chain_us * 1e-6) / 1e9
+        line["roofline"] = {"bound": "hbm", "kernel": "k_gemm_tc (one layer's chain: O-proj, gate|up, down, next QKV)",
+                            "achieved": ach, "peak": pk["hbm_gbs"], "peak_kind": pk_kind + " copy bandwidth",
+                            "unit": "GB/s", "frac": ach / pk["hbm_gbs"], "traffic": CHAIN_TRAFFIC_BYTES,
+                            "algorithmic_bytes": chain_bytes, "us_per_launch": chain_us,
+                            "launches_per_step": shape.n_layers, "share_of_step": chain_us * shape.n_layers / (ms_step * 1e3)}
+    else:
+        line["roofline"] = dict(line["step_roofline"], kernel="pass_step graph", traffic=None)
     if not args.no_cpu_baseline and world == 1:
         nl = 2 if shape.n_layers > 2 else shape.n_layers
         w_small = small_weights_from(w, nl)

@@ -211,8 +211,10 @@ int pass_debug_linear(pass_ctx *ctx, int which, int layer, const float *x_device
 /*
  * Time that kernel: n_launches launches back to back on the context's stream, cycling over the
  * layers so that every launch streams different weights from HBM (CUDA events; one untimed pass
- * over the layers first).  which as above, except 7.  Inputs are whatever the activation buffer
- * holds.  *ms_total receives the elapsed milliseconds.  Synchronises.
+ * over the layers first).  which as above, except 7; which = 9 times the step's dominant launch, the
+ * chain O-projection -> gate|up -> down -> next layer's QKV of layers 0, 1, ... (it overwrites the
+ * residual stream and row 0.. of sequence 0's cache: re-run pass_prefill afterwards).  Inputs are
+ * whatever the activation buffers hold.  *ms_total receives the elapsed milliseconds.  Synchronises.
  */
 int pass_debug_time_linear(pass_ctx *ctx, int which, int R, int n_launches, float *ms_total);
 

@@ -255,7 +255,10 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
     lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-__device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[8]) {
+// hv_pre: for kEpiResid the caller may hand in the residual values h[c0..c0+7][n] it has already
+// loaded (so that this trip to L2 overlaps with another); nullptr = load them here.
+__device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[8],
+                                          const float* hv_pre = nullptr) {
     const int L = ec.lane_in_tile;
     if (p.epi == kEpiLogits) {
         const int n = tile * kTileN + L;
@@ -301,7 +304,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         float ss[8], hv[8];
 #pragma unroll
         for (int j = 0; j < 8; j++)      // all loads first: they are independent of the stores below
-            hv[j] = (c0 + j < p.R && n < d) ? __ldcg(p.h + (size_t)(c0 + j) * d + n) : 0.f;
+            hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < p.R && n < d) ? __ldcg(p.h + (size_t)(c0 + j) * d + n) : 0.f);
 #pragma unroll
         for (int j = 0; j < 8; j++) {
             const int r = c0 + j;
@@ -419,10 +422,31 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
     __shared__ float s_x[128 * 9];
+    // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
+    // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
+    constexpr int kPieceCache = 16;
+    __shared__ Piece s_piece[kMaxOps][kPieceCache];
+    __shared__ int s_piece_ok[kMaxOps][kPieceCache];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = cp.stages;
     const int G = gridDim.x, cta = blockIdx.x;
+    if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxOps * kPieceCache) {
+        const int oi = (threadIdx.x - 128) / kPieceCache, it = (threadIdx.x - 128) % kPieceCache;
+        Piece pc;
+        pc.tile = pc.kb0 = pc.kb1 = pc.n_pieces = pc.index = pc.slot = 0;
+        const bool v = oi < cp.n_ops && get_piece(cp.op[oi], cta, G, it, pc);
+        s_piece[oi][it] = pc;
+        s_piece_ok[oi][it] = v ? 1 : 0;
+    }
+    auto fetch_piece = [&](int oi, int it, Piece& out) -> bool {
+        if (it < kPieceCache) {
+            if (!s_piece_ok[oi][it]) return false;
+            out = s_piece[oi][it];
+            return true;
+        }
+        return get_piece(cp.op[oi], cta, G, it, out);
+    };
     const uint32_t stage_bytes = kATileBytes + cp.npad * 128;
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_u32(&s_bars[0]), bar_empty = bar_full + 8 * 16;
@@ -463,7 +487,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
                 const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
-                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
                     weight_box(p, maps.m[oi], pc.tile, 0, m, y);
@@ -496,7 +520,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
                 }
                 PASS_TRACE(oi, 0);
-                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++) {
+                for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
                     weight_box(p, maps.m[oi], pc.tile, 1, m, y);
@@ -529,7 +553,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             bool stop = false;
             for (int oi = 0; !stop && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
-                for (int it = 0; !stop && get_piece(p, cta, G, it, pc); it++) {
+                for (int it = 0; !stop && fetch_piece(oi, it, pc); it++) {
                     // rows of the tile: plain = 128 rows of one matrix; interleaved = 64 rows of two
                     const char* base0; const char* base1; int row0, nrows0, nrows1;
                     if (p.interleave) {
@@ -571,7 +595,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
                 bool first = true;
-                for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++, pidx++) {
+                for (int it = 0; ok && fetch_piece(oi, it, pc); it++, pidx++) {
                     const int buf = pidx & 1;
                     if (!mbar_wait(bar_acce + 8 * buf, ((pidx >> 1) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
                     tc_fence_after();
@@ -627,7 +651,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             epi_bar();
             const size_t slot_floats = (size_t)p.rh * kTileN;
             const bool signal = oi + 1 < cp.n_ops;   // a later GEMM of the chain waits for this one's tiles
-            for (int it = 0; ok && get_piece(p, cta, G, it, pc); it++, pidx++) {
+            for (int it = 0; ok && fetch_piece(oi, it, pc); it++, pidx++) {
                 const int buf = pidx & 1;
                 // each thread waits for itself; the outcome is made uniform before any barrier is used
                 if (!mbar_wait(bar_accf + 8 * buf, (pidx >> 1) & 1, &s_abort, cp.status)) *(volatile int*)&s_epi_fail = 1;
@@ -678,6 +702,47 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         const long long ts = (long long)pc.tile * p.kb_per_tile;
                         const int Ge = G > U ? (int)U : G;
                         const int c_first = cta - pc.index;
+                        const int slot_first = (unit_start(c_first, U, Ge) >= ts) ? 0 : 1;
+                        if (p.rh == 16) {
+                            // the common case (up to 16 rows): both 8-row halves in one pass.  The residual
+                            // values and the parts of four contributors are requested together, so the whole
+                            // reduction costs one or two trips to L2 instead of one per half and contributor group.
+                            const int n = pc.tile * kTileN + ec.lane_in_tile;
+                            float hv[2][8];
+                            if (p.epi == kEpiResid) {
+#pragma unroll
+                                for (int j = 0; j < 16; j++)
+                                    hv[j >> 3][j & 7] = (j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
+                            }
+                            float acc[2][8];
+#pragma unroll
+                            for (int j = 0; j < 16; j++) acc[j >> 3][j & 7] = 0.f;
+                            for (int q0 = 0; q0 < pc.n_pieces; q0 += 4) {
+                                float4 v[4][4];
+#pragma unroll
+                                for (int qq = 0; qq < 4; qq++) {
+                                    const int qi = min(q0 + qq, pc.n_pieces - 1);
+                                    const int cq = c_first + qi;
+                                    const int slot = qi == 0 ? slot_first : 0;
+                                    const float4* src = reinterpret_cast<const float4*>(
+                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * 16);
+#pragma unroll
+                                    for (int f = 0; f < 4; f++) v[qq][f] = __ldcg(src + f);
+                                }
+#pragma unroll
+                                for (int qq = 0; qq < 4; qq++) {
+                                    if (q0 + qq < pc.n_pieces) {
+#pragma unroll
+                                        for (int f = 0; f < 4; f++) {
+                                            acc[f >> 1][(f & 1) * 4 + 0] += v[qq][f].x; acc[f >> 1][(f & 1) * 4 + 1] += v[qq][f].y;
+                                            acc[f >> 1][(f & 1) * 4 + 2] += v[qq][f].z; acc[f >> 1][(f & 1) * 4 + 3] += v[qq][f].w;
+                                        }
+                                    }
+                                }
+                            }
+                            epi_store(p, ec, pc.tile, 0, acc[0], p.epi == kEpiResid ? hv[0] : nullptr);
+                            epi_store(p, ec, pc.tile, 8, acc[1], p.epi == kEpiResid ? hv[1] : nullptr);
+                        } else
                         for (int c0 = 0; c0 < p.rh; c0 += 8) {
                             float acc[8];
 #pragma unroll
@@ -688,9 +753,10 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                 float4 v[8][2];
 #pragma unroll
                                 for (int qq = 0; qq < 8; qq++) {
-                                    const int cq = c_first + min(q0 + qq, pc.n_pieces - 1);
-                                    const long long sq = unit_start(cq, U, Ge);
-                                    const int slot = (sq >= ts) ? 0 : 1;   // piece begins at the CTA's own start?
+                                    const int qi = min(q0 + qq, pc.n_pieces - 1);
+                                    const int cq = c_first + qi;
+                                    // every contributor but the first starts its own range inside this tile
+                                    const int slot = qi == 0 ? slot_first : 0;
                                     const float4* src = reinterpret_cast<const float4*>(
                                         p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * p.rh + c0);
                                     v[qq][0] = __ldcg(src);

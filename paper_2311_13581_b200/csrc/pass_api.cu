@@ -384,46 +384,89 @@ static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
     c->launches++;
 }
 
+// GEMMs of the decoder layers as chain entries.
+static void fill_weights(GemmParams& p, const void* w0, const void* w1, const void* w2, int rows, int ld) {
+    p.w_base[0] = w0; p.w_base[1] = w1; p.w_base[2] = w2;
+    p.w_rows[0] = p.w_rows[1] = p.w_rows[2] = rows;
+    p.w_ld = ld;
+}
+static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l) {
+    typedef __nv_bfloat16 bf;
+    const int d = c->md.d, dt = d / kTileN;
+    ChainOp o;
+    o.p = gemm_base(c, R, npad, d, 3 * dt, 3 * d, kEpiQKV);
+    o.p.seg_tiles0 = o.p.seg_tiles1 = dt;
+    o.p.sumsq_in = c->d_sumsq_a; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
+    o.p.q_out = c->d_q_out; o.p.rope_cs = c->d_cs; o.p.row_seq = c->d_row_seq; o.p.row_pos = c->d_row_pos;
+    o.p.layer = l; o.p.kc = (bf*)c->kv_k; o.p.vc = (bf*)c->kv_v;
+    fill_weights(o.p, c->wq[l], c->wk[l], c->wv[l], d, d);
+    o.a0 = c->tm_wq[l]; o.a1 = c->tm_wk[l]; o.a2 = c->tm_wv[l]; o.b = bm->xn;
+    return o;
+}
+// O-projection -> gate|up -> down of layer l, then the next layer's QKV, or the output head (head = true)
+// after the last layer, or nothing.  Returns the number of entries written.
+static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l, bool head, ChainOp* ch) {
+    typedef __nv_bfloat16 bf;
+    const ModelDims& md = c->md;
+    const int d = md.d, f = md.f, dt = d / kTileN;
+    int n = 0;
+    {   // attention output projection + residual; prepares the input of the feed-forward norm
+        ChainOp& o = ch[n++];
+        o.p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
+        o.p.h = c->d_h; o.p.gain_next = (const bf*)c->norm_ffn[l]; o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_b;
+        fill_weights(o.p, c->wo[l], c->wo[l], c->wo[l], d, d);
+        o.a0 = o.a1 = o.a2 = c->tm_wo[l]; o.b = bm->attn;
+    }
+    {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
+        ChainOp& o = ch[n++];
+        o.p = gemm_base(c, R, npad, d, (f + 63) / 64, f, kEpiSwiGLU);
+        o.p.interleave = 1;
+        o.p.sumsq_in = c->d_sumsq_b; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
+        o.p.act_out = c->d_act_bf;
+        fill_weights(o.p, c->wg[l], c->wu[l], c->wu[l], f, d);
+        o.a0 = c->tm_wg[l]; o.a1 = o.a2 = c->tm_wu[l]; o.b = bm->xn;
+    }
+    {   // down projection + residual; prepares the input of the next norm
+        ChainOp& o = ch[n++];
+        o.p = gemm_base(c, R, npad, f, dt, d, kEpiResid);
+        o.p.h = c->d_h;
+        o.p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
+        o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_a;
+        fill_weights(o.p, c->wd[l], c->wd[l], c->wd[l], d, f);
+        o.a0 = o.a1 = o.a2 = c->tm_wd[l]; o.b = bm->act;
+    }
+    if (l + 1 < md.n_layers) {
+        ch[n++] = op_qkv(c, R, npad, bm, l + 1);
+    } else if (head) {
+        ChainOp& o = ch[n++];
+        o.p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
+        o.p.sumsq_in = c->d_sumsq_a; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
+        o.p.logits = c->d_logits;
+        fill_weights(o.p, c->lm_head, c->lm_head, c->lm_head, md.V, d);
+        o.a0 = o.a1 = o.a2 = c->tm_lm; o.b = bm->xn;
+    }
+    return n;
+}
+
+static void launch_ops(pass_ctx* c, ChainOp* ch, int n) {
+    if (getenv("PASS_NO_CHAIN")) for (int j = 0; j < n; j++) launch_chain(c, ch + j, 1);
+    else launch_chain(c, ch, n);
+}
+
 // R rows = n_seq sequences x M rows each (M = R when n_seq == 1).
 static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
     const ModelDims& md = c->md;
-    const int d = md.d, f = md.f, npad = npad_for(R), rh = npad / 2;
+    const int d = md.d, npad = npad_for(R), rh = npad / 2;
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     typedef __nv_bfloat16 bf;
     LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
     LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
-    const int dt = d / kTileN;
-    const bool chained = getenv("PASS_NO_CHAIN") == nullptr;
     ChainOp chain[kMaxOps];
-    int n_chain = 0;
-    auto flush = [&]() {
-        if (n_chain == 0) return;
-        if (chained) launch_chain(c, chain, n_chain);
-        else for (int j = 0; j < n_chain; j++) launch_chain(c, chain + j, 1);
-        n_chain = 0;
-    };
-    auto add = [&](GemmParams p, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
-                   const CUtensorMap& b, const void* w0, const void* w1, const void* w2, int rows, int ld) {
-        p.w_base[0] = w0; p.w_base[1] = w1; p.w_base[2] = w2;
-        p.w_rows[0] = p.w_rows[1] = p.w_rows[2] = rows;
-        p.w_ld = ld;
-        chain[n_chain].p = p; chain[n_chain].a0 = a0; chain[n_chain].a1 = a1; chain[n_chain].a2 = a2;
-        chain[n_chain].b = b;
-        n_chain++;
-    };
-    auto qkv = [&](int l) {   // q | k | v
-        GemmParams p = gemm_base(c, R, npad, d, 3 * dt, 3 * d, kEpiQKV);
-        p.seg_tiles0 = p.seg_tiles1 = dt;
-        p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
-        p.q_out = c->d_q_out; p.rope_cs = c->d_cs; p.row_seq = c->d_row_seq; p.row_pos = c->d_row_pos;
-        p.layer = l; p.kc = (bf*)c->kv_k; p.vc = (bf*)c->kv_v;
-        add(p, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], bm->xn, c->wq[l], c->wk[l], c->wv[l], d, d);
-    };
     // Kernels of a step: QKV_0 | per layer: attention, then ONE launch running
     // O-projection -> gate|up -> down -> (next layer's QKV, or the output head after the last layer).
-    qkv(0);
-    flush();
+    chain[0] = op_qkv(c, R, npad, bm, 0);
+    launch_ops(c, chain, 1);
     for (int l = 0; l < md.n_layers; l++) {
         const int M = R / n_seq;
         if (M <= 32) {
@@ -441,34 +484,7 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
         } else {
             LAUNCH(c, (k_attn_simple<bf, 64, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
         }
-        {   // attention output projection + residual; prepares the input of the feed-forward norm
-            GemmParams p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
-            p.h = c->d_h; p.gain_next = (const bf*)c->norm_ffn[l]; p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_b;
-            add(p, c->tm_wo[l], c->tm_wo[l], c->tm_wo[l], bm->attn, c->wo[l], c->wo[l], c->wo[l], d, d);
-        }
-        {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
-            GemmParams p = gemm_base(c, R, npad, d, (f + 63) / 64, f, kEpiSwiGLU);
-            p.interleave = 1;
-            p.sumsq_in = c->d_sumsq_b; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
-            p.act_out = c->d_act_bf;
-            add(p, c->tm_wg[l], c->tm_wu[l], c->tm_wu[l], bm->xn, c->wg[l], c->wu[l], c->wu[l], f, d);
-        }
-        {   // down projection + residual; prepares the input of the next norm
-            GemmParams p = gemm_base(c, R, npad, f, dt, d, kEpiResid);
-            p.h = c->d_h;
-            p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
-            p.xn_out = c->d_xn_bf; p.sumsq_out = c->d_sumsq_a;
-            add(p, c->tm_wd[l], c->tm_wd[l], c->tm_wd[l], bm->act, c->wd[l], c->wd[l], c->wd[l], d, f);
-        }
-        if (l + 1 < md.n_layers) {
-            qkv(l + 1);
-        } else if (head) {
-            GemmParams p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
-            p.sumsq_in = c->d_sumsq_a; p.n_parts_in = dt; p.inv_d_in = 1.f / d;
-            p.logits = c->d_logits;
-            add(p, c->tm_lm, c->tm_lm, c->tm_lm, bm->xn, c->lm_head, c->lm_head, c->lm_head, md.V, d);
-        }
-        flush();
+        launch_ops(c, chain, build_layer_chain(c, R, npad, bm, l, head, chain));
     }
     return PASS_OK;
 }
@@ -1034,22 +1050,38 @@ int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, 
 }
 
 int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float* ms_total) {
-    if (!c || !ms_total || which < 0 || which > 8 || which == 7 || R < 1 || R > kMaxRows || n_launches < 1)
+    if (!c || !ms_total || which < 0 || which > 9 || which == 7 || R < 1 || R > kMaxRows || n_launches < 1)
         return PASS_ERR_INVALID_ARG;
     if (!c->weights_loaded || !c->use_tc) return PASS_ERR_STATE;
     const int N = which == 8 ? ((c->md.f + 63) / 64) * 128 : (which == 4 || which == 5 ? c->md.f : c->md.d);
-    if (N > c->md.V) return PASS_ERR_CAPACITY;          // results land in the logits buffer
+    if (which != 9 && N > c->md.V) return PASS_ERR_CAPACITY;          // results land in the logits buffer
+    if (which == 9 && c->md.n_layers < 2) return PASS_ERR_INVALID_ARG;
     if (c->pending_collect) {
         const int rc = pass_step_collect(c, nullptr, nullptr);
         if (rc != PASS_OK) return rc;
     }
+    const int npad = npad_for(R), nl = c->md.n_layers;
+    const pass_ctx::BMaps* bm = get_bmaps(c, npad);
+    if (!bm) return PASS_ERR_CUDA;
+    auto one = [&](int i) {
+        if (which == 9) {          // the step's dominant launch: O-proj -> gate|up -> down -> next layer's QKV
+            ChainOp chain[kMaxOps];
+            const int l = i % (nl - 1);
+            launch_ops(c, chain, build_layer_chain(c, R, npad, bm, l, false, chain));
+        } else {
+            enqueue_debug_linear(c, which, i % nl, R, c->d_logits);
+        }
+    };
+    if (which == 9) {              // rows at position 0 of sequence 0: the QKV epilogue needs valid row tables
+        CUDA_TRY(cudaMemsetAsync(c->d_row_seq, 0, sizeof(int) * kMaxRows, c->stream));
+        CUDA_TRY(cudaMemsetAsync(c->d_row_pos, 0, sizeof(int) * kMaxRows, c->stream));
+    }
     cudaEvent_t e0, e1;
     CUDA_TRY(cudaEventCreate(&e0));
     CUDA_TRY(cudaEventCreate(&e1));
-    for (int i = 0; i < std::min(n_launches, c->md.n_layers); i++)        // warm-up pass
-        enqueue_debug_linear(c, which, i % c->md.n_layers, R, c->d_logits);
+    for (int i = 0; i < std::min(n_launches, nl); i++) one(i);        // warm-up pass
     CUDA_TRY(cudaEventRecord(e0, c->stream));
-    for (int i = 0; i < n_launches; i++) enqueue_debug_linear(c, which, i % c->md.n_layers, R, c->d_logits);
+    for (int i = 0; i < n_launches; i++) one(i);
     CUDA_TRY(cudaEventRecord(e1, c->stream));
     CUDA_TRY(cudaGetLastError());
     CUDA_TRY(cudaStreamSynchronize(c->stream));
