@@ -36,6 +36,9 @@ constexpr int kBlockK = 64;
 constexpr int kGemmThreads = 256;
 constexpr int kATileBytes = kTileN * kBlockK * 2;       // 16 KB
 constexpr long long kWaitCycles = 400000000LL;          // ~0.2 s at 2 GHz
+// Upper limit (ns) for which one mbarrier.try_wait may park the thread in hardware.  A parked waiter
+// takes no issue slots from the epilogue warps on its scheduler and wakes as soon as the phase completes.
+constexpr uint32_t kSuspendHintNs = 20000;
 
 enum GemmEpilogue { kEpiLogits = 0, kEpiQKV = 1, kEpiResid = 2, kEpiSwiGLU = 3 };
 
@@ -92,9 +95,9 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok;
 }
 // Bounded wait: false when the CTA is giving up (another role timed out, or this wait did).
