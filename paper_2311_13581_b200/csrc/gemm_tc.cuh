@@ -215,6 +215,7 @@ struct Piece {
     int tile, kb0, kb1;      // k-blocks [kb0, kb1) of the tile
     int n_pieces, index;     // how many CTAs share the tile, and which of them this is (k order)
     int slot;                // partial slot of this CTA (0 = its first piece, 1 = a later one)
+    int first_slot;          // slot used by the tile's first contributor (the only one that may have begun earlier)
 };
 
 __device__ __forceinline__ long long unit_start(long long c, long long U, long long G) { return c * U / G; }
@@ -242,6 +243,7 @@ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int
     out.n_pieces = c_last - c_first + 1;
     out.index = c - c_first;
     out.slot = (a == s) ? 0 : 1;
+    out.first_slot = (unit_start(c_first, U, G) >= ts) ? 0 : 1;
     return true;
 }
 
@@ -320,7 +322,14 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
                 p.xn_out[(size_t)r * d + n] = hi;
                 p.xn_out[(size_t)(p.xn_lo_row0 + r) * d + n] = lo;
             }
-            ss[j] = warp_sum(hn * hn);
+            ss[j] = hn * hn;
+        }
+        // eight butterfly reductions side by side: each level issues eight independent shuffles, so the
+        // shuffle latency is paid five times, not forty
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int j = 0; j < 8; j++) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], o);
         }
         epi_bar();                                  // s_x free
         if (lane == 0) {
@@ -437,7 +446,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     if (threadIdx.x >= 128 && threadIdx.x < 128 + kMaxOps * kPieceCache) {
         const int oi = (threadIdx.x - 128) / kPieceCache, it = (threadIdx.x - 128) % kPieceCache;
         Piece pc;
-        pc.tile = pc.kb0 = pc.kb1 = pc.n_pieces = pc.index = pc.slot = 0;
+        pc.tile = pc.kb0 = pc.kb1 = pc.n_pieces = pc.index = pc.slot = pc.first_slot = 0;
         const bool v = oi < cp.n_ops && get_piece(cp.op[oi], cta, G, it, pc);
         s_piece[oi][it] = pc;
         s_piece_ok[oi][it] = v ? 1 : 0;
@@ -705,7 +714,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         const long long ts = (long long)pc.tile * p.kb_per_tile;
                         const int Ge = G > U ? (int)U : G;
                         const int c_first = cta - pc.index;
-                        const int slot_first = (unit_start(c_first, U, Ge) >= ts) ? 0 : 1;
+                        const int slot_first = pc.first_slot;
                         if (p.rh == 16) {
                             // the common case (up to 16 rows): both 8-row halves in one pass.  The residual
                             // values and the parts of four contributors are requested together, so the whole
