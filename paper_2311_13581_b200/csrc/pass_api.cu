@@ -252,7 +252,7 @@ static int gemm_stages(int npad) {
         const int s = atoi(e);
         if (s >= 2 && s <= 16 && (size_t)s * stage + 1024 <= 225 * 1024) return s;
     }
-    int s = (112 * 1024 - 1024) / stage;
+    int s = (122 * 1024 - 1024) / stage;   // leaves room for one attention CTA (96 KB) beside it
     if (s < 4) s = std::min(4, (220 * 1024) / stage);
     return std::max(2, std::min(16, s));
 }
