@@ -134,6 +134,19 @@ def oracle_sample(shape, w_cpu_small, n_small_layers, k, ctx_len, reps):
     return per_step, po.num_threads(), desc
 
 
+def aggregate_replicas(ms_total, e2e_ms, tokens, tok_e2e, world, device):
+    """Whole-job numbers from per-replica ones: the path has no exchange step, so N GPUs run N
+    independent replicas; time is the MAX over ranks, tokens are the SUM (weak scaling)."""
+    if world <= 1:
+        return ms_total, e2e_ms, tokens, tok_e2e
+    import torch.distributed as dist
+    t = torch.tensor([ms_total, e2e_ms, float(tokens), float(tok_e2e)], dtype=torch.float64, device=device)
+    tmax, tsum = t.clone(), t.clone()
+    dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+    return float(tmax[0]), float(tmax[1]), float(tsum[2]), float(tsum[3])
+
+
 def small_weights_from(w, n_layers):
     out = {}
     for k, v in w.items():
@@ -254,16 +267,7 @@ def main():
         n_chain = 64
         chain_us = min(ctx.debug_time_linear(9, B * (1 + 2 * k), n_chain) for _ in range(3)) * 1e3 / n_chain
 
-    t = torch.tensor([ms_total, e2e_s * 1e3, float(tokens), float(tok_e2e)], dtype=torch.float64, device=dev)
-    if world > 1:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms_total, e2e_ms = float(tmax[0]), float(tmax[1])
-        tokens, tok_e2e = float(tsum[2]), float(tsum[3])
-    else:
-        e2e_ms = e2e_s * 1e3
+    ms_total, e2e_ms, tokens, tok_e2e = aggregate_replicas(ms_total, e2e_s * 1e3, tokens, tok_e2e, world, dev)
     if rank != 0:
         return
 

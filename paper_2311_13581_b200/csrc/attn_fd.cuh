@@ -105,8 +105,10 @@ k_attn_fd(const AttnParams p) {
         }
     };
 
-    // query fragments (A operand), scaled by log2(e)/sqrt(d_head) so that exp2 can be used
-    uint32_t qf[DH / 16][4];
+    // query fragments (A operand), scaled by log2(e)/sqrt(d_head) so that exp2 can be used.  Queries and
+    // probabilities are carried as bf16 hi + bf16 lo (two MMAs each): a single bf16 rounding of q or p
+    // (2^-9 relative) would go straight into the output, since the output is a sum of the same terms.
+    uint32_t qf[DH / 16][4], qfl[DH / 16][4];
     {
         const float sc = 1.4426950408889634f * rsqrtf((float)DH);
         const int i0 = mt * 16 + g, i1 = i0 + 8;
@@ -118,10 +120,14 @@ k_attn_fd(const AttnParams p) {
             float2 a = make_float2(0.f, 0.f), bq = a, c2 = a, d2 = a;
             if (i0 < M) { a = *reinterpret_cast<const float2*>(q0 + c); c2 = *reinterpret_cast<const float2*>(q0 + c + 8); }
             if (i1 < M) { bq = *reinterpret_cast<const float2*>(q1 + c); d2 = *reinterpret_cast<const float2*>(q1 + c + 8); }
-            qf[ks][0] = pack_bf16(a.x * sc, a.y * sc);
-            qf[ks][1] = pack_bf16(bq.x * sc, bq.y * sc);
-            qf[ks][2] = pack_bf16(c2.x * sc, c2.y * sc);
-            qf[ks][3] = pack_bf16(d2.x * sc, d2.y * sc);
+            const float2 f4[4] = {a, bq, c2, d2};
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const float x = f4[e].x * sc, y = f4[e].y * sc;
+                const __nv_bfloat162 hi = __floats2bfloat162_rn(x, y);
+                qf[ks][e] = *reinterpret_cast<const uint32_t*>(&hi);
+                qfl[ks][e] = pack_bf16(x - __low2float(hi), y - __high2float(hi));
+            }
         }
     }
 
@@ -160,6 +166,8 @@ k_attn_fd(const AttnParams p) {
                     ldsm_x4(kS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
                     mma_bf16_16816(s[0], qf[ks], r[0], r[1]);
                     mma_bf16_16816(s[1], qf[ks], r[2], r[3]);
+                    mma_bf16_16816(s[0], qfl[ks], r[0], r[1]);
+                    mma_bf16_16816(s[1], qfl[ks], r[2], r[3]);
                 }
             }
             // causal mask: row i sees key j iff j <= len + i
@@ -199,11 +207,16 @@ k_attn_fd(const AttnParams p) {
             l_run[1] = l_run[1] * c1 + ps1;
 #pragma unroll
             for (int n = 0; n < DH / 8; n++) { o[n][0] *= c0; o[n][1] *= c0; o[n][2] *= c1; o[n][3] *= c1; }
-            uint32_t pa[4];
-            pa[0] = pack_bf16(s[0][0], s[0][1]);
-            pa[1] = pack_bf16(s[0][2], s[0][3]);
-            pa[2] = pack_bf16(s[1][0], s[1][1]);
-            pa[3] = pack_bf16(s[1][2], s[1][3]);
+            uint32_t pa[4], pl[4];
+            {
+                const float ps[4][2] = {{s[0][0], s[0][1]}, {s[0][2], s[0][3]}, {s[1][0], s[1][1]}, {s[1][2], s[1][3]}};
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(ps[e][0], ps[e][1]);
+                    pa[e] = *reinterpret_cast<const uint32_t*>(&hi);
+                    pl[e] = pack_bf16(ps[e][0] - __low2float(hi), ps[e][1] - __high2float(hi));
+                }
+            }
             {
                 const int mi = lane >> 3, rr = lane & 7;
                 const int key = key0 + (mi & 1) * 8 + rr;
@@ -214,6 +227,8 @@ k_attn_fd(const AttnParams p) {
                     ldsm_x4_trans(vS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
                     mma_bf16_16816(o[2 * np], pa, r[0], r[1]);
                     mma_bf16_16816(o[2 * np + 1], pa, r[2], r[3]);
+                    mma_bf16_16816(o[2 * np], pl, r[0], r[1]);
+                    mma_bf16_16816(o[2 * np + 1], pl, r[2], r[3]);
                 }
             }
         }
