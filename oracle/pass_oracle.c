@@ -30,6 +30,7 @@
 typedef struct {
     int n_layers, d_model, n_heads, d_head, d_ffn, vocab;
     int wdtype;                 /* 0 = float32, 1 = bfloat16 (uint16 bit patterns) */
+    int kvdtype;                /* how a K/V row is stored: 0 = as computed (float64), 1 = rounded to bfloat16 */
     double rms_eps, rope_theta;
     const void *lm_head, *final_norm;
     const void *const *wq, *const *wk, *const *wv, *const *wo;
@@ -43,6 +44,20 @@ static inline double w_at(const void *w, int dtype, size_t i) {
     float f;
     memcpy(&f, &bits, 4);
     return (double)f;
+}
+
+/* Nearest bfloat16 (sign, 8 exponent bits, 7 fraction bits), ties to even, of a double in bfloat16's
+ * normal range; zero, and anything outside that range, is returned as it is. */
+static inline double to_bf16(double x) {
+    const double ax = fabs(x);
+    if (!(ax >= 0x1p-126 && ax < 0x1p127)) return x;
+    uint64_t b;
+    memcpy(&b, &x, 8);
+    const uint64_t drop = 52 - 7;                      /* fraction bits that do not fit */
+    b += (((uint64_t)1 << (drop - 1)) - 1) + ((b >> drop) & 1);
+    b &= ~(((uint64_t)1 << drop) - 1);
+    memcpy(&x, &b, 8);
+    return x;
 }
 
 /* y[r][o] = sum_k x[r][k] * W[o][k]   (W is [n_out][n_in] row-major) */
@@ -175,8 +190,12 @@ int oracle_forward(const oracle_model *m, const double *x_in, int n_rows, int po
         for (int r = 0; r < n_rows; r++) {
             rope(m, q + (size_t)r * d, pos0 + r);
             rope(m, kk + (size_t)r * d, pos0 + r);
-            memcpy(kc + (size_t)(pos0 + r) * d, kk + (size_t)r * d, sizeof(double) * d);
-            memcpy(vc + (size_t)(pos0 + r) * d, vv + (size_t)r * d, sizeof(double) * d);
+            /* the cache holds what its storage format can hold; attention reads the cache */
+            for (int i = 0; i < d; i++) {
+                const double kx = kk[(size_t)r * d + i], vx = vv[(size_t)r * d + i];
+                kc[(size_t)(pos0 + r) * d + i] = m->kvdtype == 1 ? to_bf16(kx) : kx;
+                vc[(size_t)(pos0 + r) * d + i] = m->kvdtype == 1 ? to_bf16(vx) : vx;
+            }
         }
         attention(m, q, kc, vc, n_rows, pos0, o);
         linear(m, m->wo[l], d, d, o, n_rows, t);

@@ -62,7 +62,7 @@ def build_oracle(force: bool = False) -> str:
 
 class _CModel(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
-                ("n_layers", "d_model", "n_heads", "d_head", "d_ffn", "vocab", "wdtype")] + \
+                ("n_layers", "d_model", "n_heads", "d_head", "d_ffn", "vocab", "wdtype", "kvdtype")] + \
                [("rms_eps", ctypes.c_double), ("rope_theta", ctypes.c_double),
                 ("lm_head", ctypes.c_void_p), ("final_norm", ctypes.c_void_p)] + \
                [(n, ctypes.POINTER(ctypes.c_void_p)) for n in
@@ -103,9 +103,15 @@ class TransformerBackend:
     causal mask, look-ahead rows appended after the real tokens - Look-ahead
     embeddings) and returns float64 logits [len(rows), vocab].  Whatever the cache
     held at positions >= pos0 is overwritten: that is the rollback.
+
+    ``kv_dtype`` is the storage format of the cache.  The paper does not fix one
+    (Experiments, setup), so the default "f64" keeps every row as computed.
+    "bf16" models a bfloat16 cache: each K/V row is rounded (nearest, ties to even)
+    when it is stored, and attention reads the stored values - the arithmetic stays
+    float64.  That isolates the one error a bf16 cache makes by construction.
     """
 
-    def __init__(self, shape, weights, kv_capacity: int):
+    def __init__(self, shape, weights, kv_capacity: int, kv_dtype: str = "f64"):
         import torch
         self.shape = shape
         self.w = weights
@@ -123,6 +129,7 @@ class TransformerBackend:
         cm.n_layers, cm.d_model, cm.n_heads = shape.n_layers, d, shape.n_heads
         cm.d_head, cm.d_ffn, cm.vocab = shape.d_head, shape.d_ffn, shape.vocab
         cm.wdtype = 0 if dt == torch.float32 else 1
+        cm.kvdtype = {"f64": 0, "bf16": 1}[kv_dtype]
         cm.rms_eps, cm.rope_theta = float(shape.rms_eps), float(shape.rope_theta)
         cm.lm_head = weights["lm_head"].data_ptr()
         cm.final_norm = weights["final_norm"].data_ptr()
@@ -169,7 +176,7 @@ class Pieces:
         cm = _CModel()
         cm.n_layers, cm.d_model, cm.n_heads = shape.n_layers, shape.d_model, shape.n_heads
         cm.d_head, cm.d_ffn, cm.vocab = shape.d_head, shape.d_ffn, shape.vocab
-        cm.wdtype = wdtype
+        cm.wdtype, cm.kvdtype = wdtype, 0
         cm.rms_eps, cm.rope_theta = float(shape.rms_eps), float(shape.rope_theta)
         self._cm, self._lib, self.shape = cm, _load(), shape
 

@@ -134,7 +134,7 @@ def test_attention_closed_forms_and_library():
 
 
 # ---------------------------------------------------------------- whole forward
-def _torch_forward(shape, w, x, pos0, kc, vc):
+def _torch_forward(shape, w, x, pos0, kc, vc, store=lambda t: t):
     """float64 transcription with library matmul / softmax (a cross-check, all rows at once)."""
     W = lambda t: t.double()
     d, H, dh = shape.d_model, shape.n_heads, shape.d_head
@@ -155,7 +155,7 @@ def _torch_forward(shape, w, x, pos0, kc, vc):
     for l in range(shape.n_layers):
         a = norm(h, w["norm_attn"][l])
         q, k, v = rope(a @ W(w["wq"][l]).T), rope(a @ W(w["wk"][l]).T), a @ W(w["wv"][l]).T
-        kc[l][pos0:pos0 + n], vc[l][pos0:pos0 + n] = k, v
+        kc[l][pos0:pos0 + n], vc[l][pos0:pos0 + n] = store(k), store(v)
         K = kc[l][:pos0 + n].reshape(-1, H, dh).transpose(0, 1)
         V = vc[l][:pos0 + n].reshape(-1, H, dh).transpose(0, 1)
         s = q.reshape(n, H, dh).transpose(0, 1) @ K.transpose(1, 2) / math.sqrt(dh)
@@ -182,6 +182,41 @@ def test_forward_against_torch_float64_transcription(tiny_weights):
     np.testing.assert_allclose(z0, t0, rtol=0, atol=1e-11)
     np.testing.assert_allclose(z1, t1, rtol=0, atol=1e-11)
     assert np.abs(z1).max() > 0.1                    # not a vacuous comparison
+
+
+def _nearest_bf16(t):
+    """bfloat16 has 8 significant bits: x = m 2^e with m in [0.5, 1) -> rint(256 m) 2^(e-8), ties to even."""
+    m, e = np.frexp(t.numpy())
+    return torch.from_numpy(np.ldexp(np.rint(m * 256.0), e - 8))
+
+
+def test_bf16_cache_stores_rounded_rows_and_attention_reads_them(tiny_weights):
+    prompt = si.make_prompt(TINY, 20)
+    rows = [("tok", t) for t in prompt[:17]]
+    rows2 = [("tok", prompt[17]), ("tok", prompt[18]), ("la", 0), ("la", 1), ("la", 2)]
+    be = po.TransformerBackend(TINY, tiny_weights, 64, kv_dtype="bf16")
+    ref = po.TransformerBackend(TINY, tiny_weights, 64)
+    z0, z1 = be.forward(rows, 0), be.forward(rows2, 17)
+    r0, r1 = ref.forward(rows, 0), ref.forward(rows2, 17)
+    # what is stored is representable in 8 significant bits, and is the nearest such value: layer 0 sees
+    # the same input in both backends, so its rows are the unrounded ones, rounded
+    for c, cr in ((be.k, ref.k), (be.v, ref.v)):
+        t = torch.from_numpy(c[:, :22])
+        assert torch.equal(t.to(torch.bfloat16).double(), t)
+        assert torch.equal(torch.from_numpy(c[0, :22]), _nearest_bf16(torch.from_numpy(cr[0, :22])))
+        assert np.all(np.abs(c[0, :22] - cr[0, :22]) <= 2.0 ** -8 * np.abs(cr[0, :22]))   # half a step: 2^-9 x / m, m >= 1/2
+    assert _nearest_bf16(torch.tensor([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -0.75, 0.0],
+                                      dtype=torch.float64)).tolist() == [1.0, 1.0 + 2.0 ** -6, -0.75, 0.0]
+    # the forward with that cache, transcribed
+    kc = torch.zeros(TINY.n_layers, 64, TINY.d_model, dtype=torch.float64)
+    vc = torch.zeros_like(kc)
+    t0 = _torch_forward(TINY, tiny_weights, be.embed(rows), 0, kc, vc, store=_nearest_bf16)
+    t1 = _torch_forward(TINY, tiny_weights, be.embed(rows2), 17, kc, vc, store=_nearest_bf16)
+    np.testing.assert_allclose(z0, t0, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(z1, t1, rtol=0, atol=1e-11)
+    # and it is a different computation from the unrounded one, by about the format's step
+    err = np.linalg.norm(z1 - r1) / np.linalg.norm(r1)
+    assert 1e-5 < err < 1e-2, err
 
 
 def test_forward_reduces_to_head_of_embedding_when_blocks_are_zero():
