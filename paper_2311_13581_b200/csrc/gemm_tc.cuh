@@ -253,6 +253,8 @@ struct EpiCtx {
     int lane_in_tile;        // 0..127
     float* s_rstd;           // [kMaxRows]
     float* s_x;              // [128][9] exchange buffer
+    const int* s_rseq;       // [kMaxRows] sequence of each token row   (kEpiQKV)
+    const int* s_rpos;       // [kMaxRows] position of each token row   (kEpiQKV)
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -262,8 +264,11 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 
 // hv_pre: for kEpiResid the caller may hand in the residual values h[c0..c0+7][n] it has already
 // loaded (so that this trip to L2 overlaps with another); nullptr = load them here.
+// g_pre / cs_pre: likewise the next norm's gain for this feature (kEpiResid) and the eight rotation pairs
+// (kEpiQKV), fetched by the caller while it was still waiting for the accumulator.
 __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[8],
-                                          const float* hv_pre = nullptr) {
+                                          const float* hv_pre = nullptr, const float* g_pre = nullptr,
+                                          const float2* cs_pre = nullptr) {
     const int L = ec.lane_in_tile;
     if (p.epi == kEpiLogits) {
         const int n = tile * kTileN + L;
@@ -282,9 +287,9 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
 #pragma unroll
         for (int j = 0; j < 8; j++) {
             const int r = min(c0 + j, p.R - 1);
-            rs[j] = __ldg(p.row_seq + r);
-            rp[j] = __ldg(p.row_pos + r);
-            cs[j] = __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
+            rs[j] = ec.s_rseq[r];
+            rp[j] = ec.s_rpos[r];
+            cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
         }
 #pragma unroll
         for (int j = 0; j < 8; j++) {
@@ -304,7 +309,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
     } else if (p.epi == kEpiResid) {
         const int d = p.n_out;
         const int n = tile * kTileN + L;
-        const float g = n < d ? __bfloat162float(p.gain_next[n]) : 0.f;
+        const float g = g_pre ? *g_pre : (n < d ? __bfloat162float(p.gain_next[n]) : 0.f);
         const int warp_q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
         float ss[8], hv[8];
 #pragma unroll
@@ -423,7 +428,7 @@ __device__ __forceinline__ void weight_box(const GemmParams& p, const CUtensorMa
     }
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __maxnreg__(168)
 k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
@@ -433,6 +438,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_last;
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
+    __shared__ int s_rseq[kMaxRows], s_rpos[kMaxRows];
     __shared__ float s_x[128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
@@ -637,6 +643,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         ec.lane_in_tile = wq * 32 + lane;
         ec.s_rstd = s_rstd;
         ec.s_x = s_x;
+        ec.s_rseq = s_rseq;
+        ec.s_rpos = s_rpos;
         const int et = (warp - 2) * 32 + lane;        // 0..127
         griddep_wait();
         int pidx = 0;
@@ -659,12 +667,28 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     rs = rsqrtf(ss * p.inv_d_in + p.eps);
                 }
                 s_rstd[r] = rs;
+                if (p.epi == kEpiQKV) { s_rseq[r] = __ldg(p.row_seq + r); s_rpos[r] = __ldg(p.row_pos + r); }
             }
             epi_bar();
             const size_t slot_floats = (size_t)p.rh * kTileN;
             const bool signal = oi + 1 < cp.n_ops;   // a later GEMM of the chain waits for this one's tiles
             for (int it = 0; ok && fetch_piece(oi, it, pc); it++, pidx++) {
                 const int buf = pidx & 1;
+                // what the epilogue of this tile reads besides the accumulator is requested now, so that
+                // the trip to L2 is over by the time the accumulator is complete
+                float g_pre = 0.f;
+                float2 cs_pre[16];
+                const bool pre = p.rh == 16 && pc.n_pieces > 1;
+                if (pre && p.epi == kEpiResid) {
+                    const int n = pc.tile * kTileN + ec.lane_in_tile;
+                    g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
+                }
+                if (pre && p.epi == kEpiQKV) {
+                    const int i2 = ((pc.tile * kTileN + ec.lane_in_tile) % p.md.dh) >> 1;
+#pragma unroll
+                    for (int j = 0; j < 16; j++)
+                        cs_pre[j] = __ldg(p.rope_cs + (size_t)min(j, p.R - 1) * (p.md.dh / 2) + i2);
+                }
                 // each thread waits for itself; the outcome is made uniform before any barrier is used
                 if (!mbar_wait(bar_accf + 8 * buf, (pidx >> 1) & 1, &s_abort, cp.status)) *(volatile int*)&s_epi_fail = 1;
                 epi_bar();
@@ -729,31 +753,35 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                             float acc[2][8];
 #pragma unroll
                             for (int j = 0; j < 16; j++) acc[j >> 3][j & 7] = 0.f;
-                            for (int q0 = 0; q0 < pc.n_pieces; q0 += 4) {
-                                float4 v[4][4];
+                            // up to six contributors per trip (the 7B/13B shapes never have more on a tile)
+                            // and only the float4s that hold real rows
+                            const int nf4 = (p.R + 3) >> 2;
+                            for (int q0 = 0; q0 < pc.n_pieces; q0 += 6) {
+                                float4 v[6][4];
 #pragma unroll
-                                for (int qq = 0; qq < 4; qq++) {
+                                for (int qq = 0; qq < 6; qq++) {
                                     const int qi = min(q0 + qq, pc.n_pieces - 1);
                                     const int cq = c_first + qi;
                                     const int slot = qi == 0 ? slot_first : 0;
                                     const float4* src = reinterpret_cast<const float4*>(
                                         p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * 16);
 #pragma unroll
-                                    for (int f = 0; f < 4; f++) v[qq][f] = __ldcg(src + f);
+                                    for (int f = 0; f < 4; f++)
+                                        v[qq][f] = (f < nf4 && q0 + qq < pc.n_pieces) ? __ldcg(src + f) : make_float4(0.f, 0.f, 0.f, 0.f);
                                 }
 #pragma unroll
-                                for (int qq = 0; qq < 4; qq++) {
-                                    if (q0 + qq < pc.n_pieces) {
+                                for (int qq = 0; qq < 6; qq++) {
 #pragma unroll
-                                        for (int f = 0; f < 4; f++) {
-                                            acc[f >> 1][(f & 1) * 4 + 0] += v[qq][f].x; acc[f >> 1][(f & 1) * 4 + 1] += v[qq][f].y;
-                                            acc[f >> 1][(f & 1) * 4 + 2] += v[qq][f].z; acc[f >> 1][(f & 1) * 4 + 3] += v[qq][f].w;
-                                        }
+                                    for (int f = 0; f < 4; f++) {
+                                        acc[f >> 1][(f & 1) * 4 + 0] += v[qq][f].x; acc[f >> 1][(f & 1) * 4 + 1] += v[qq][f].y;
+                                        acc[f >> 1][(f & 1) * 4 + 2] += v[qq][f].z; acc[f >> 1][(f & 1) * 4 + 3] += v[qq][f].w;
                                     }
                                 }
                             }
-                            epi_store(p, ec, pc.tile, 0, acc[0], p.epi == kEpiResid ? hv[0] : nullptr);
-                            epi_store(p, ec, pc.tile, 8, acc[1], p.epi == kEpiResid ? hv[1] : nullptr);
+                            epi_store(p, ec, pc.tile, 0, acc[0], p.epi == kEpiResid ? hv[0] : nullptr,
+                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs_pre : nullptr);
+                            epi_store(p, ec, pc.tile, 8, acc[1], p.epi == kEpiResid ? hv[1] : nullptr,
+                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs_pre + 8 : nullptr);
                         } else
                         for (int c0 = 0; c0 < p.rh; c0 += 8) {
                             float acc[8];
