@@ -62,6 +62,65 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Merge of the slices of one (sequence, head) by the CTA that delivered last.  NS = most slices this
+// instance handles, EB = output elements per thread and batch.  The first batch of partial outputs and
+// the (max, sum) pairs are requested together, before anything waits: for the usual case (up to 4 slices,
+// up to 12 rows of 128) the whole merge is one trip to L2.
+template <int DH, int NS, int EB>
+__device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int row0, int head, float* sm_f) {
+    const int tid = threadIdx.x, M = p.M;
+    auto load_batch = [&](int base, float (&vals)[EB][NS]) {
+#pragma unroll
+        for (int e = 0; e < EB; e++) {
+            const int idx = min(base + e * 128 + tid, M * DH - 1);
+            const int i = idx / DH, dcol = idx % DH;
+#pragma unroll
+            for (int sidx = 0; sidx < NS; sidx++)
+                vals[e][sidx] = sidx < p.n_split ? __ldcg(p.part_o + (hb + sidx * 32 + i) * DH + dcol) : 0.f;
+        }
+    };
+    float vals[EB][NS];
+    load_batch(0, vals);
+    for (int i = tid; i < M; i += 128) {
+        float2 ml[NS];
+#pragma unroll
+        for (int sidx = 0; sidx < NS; sidx++)
+            ml[sidx] = sidx < p.n_split ? __ldcg(reinterpret_cast<const float2*>(p.part_ml) + hb + sidx * 32 + i)
+                                        : make_float2(-INFINITY, 0.f);
+        float mm = -INFINITY;
+#pragma unroll
+        for (int sidx = 0; sidx < NS; sidx++) mm = fmaxf(mm, ml[sidx].x);
+        float ll = 0.f, f[NS];
+#pragma unroll
+        for (int sidx = 0; sidx < NS; sidx++) {
+            f[sidx] = ml[sidx].x == -INFINITY ? 0.f : exp2f(ml[sidx].x - mm);
+            ll += ml[sidx].y * f[sidx];
+        }
+        const float inv = 1.f / ll;
+#pragma unroll
+        for (int sidx = 0; sidx < NS; sidx++)
+            if (sidx < p.n_split) sm_f[sidx * 32 + i] = f[sidx] * inv;
+    }
+    __syncthreads();
+    for (int base = 0; base < M * DH; base += 128 * EB) {
+        if (base > 0) load_batch(base, vals);
+#pragma unroll
+        for (int e = 0; e < EB; e++) {
+            const int idx = base + e * 128 + tid;
+            if (idx < M * DH) {
+                const int i = idx / DH, dcol = idx % DH;
+                float v = 0.f;
+#pragma unroll
+                for (int sidx = 0; sidx < NS; sidx++)
+                    if (sidx < p.n_split) v += vals[e][sidx] * sm_f[sidx * 32 + i];
+                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+                p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            }
+        }
+    }
+}
+
 template <int DH, int MT>
 __global__ void __launch_bounds__(128)
 k_attn_fd(const AttnParams p) {
@@ -81,8 +140,10 @@ k_attn_fd(const AttnParams p) {
     const int M = p.M, row0 = b * M;
     const int seq = p.row_seq[row0], len = p.row_pos[row0];
     const int n_tot = len + M;
+    // keys are dealt out in granules of 16 (one warp's share of a block), so that no slice is left
+    // empty while another holds a whole block more
     int chunk = (n_tot + p.n_split - 1) / p.n_split;
-    chunk = ((chunk + kAttnBK - 1) / kAttnBK) * kAttnBK;
+    chunk = ((chunk + 15) / 16) * 16;
     const int k_begin = split * chunk;
     const int k_end = min(n_tot, k_begin + chunk);
     const int nb = k_end > k_begin ? (k_end - k_begin + kAttnBK - 1) / kAttnBK : 0;
@@ -104,6 +165,14 @@ k_attn_fd(const AttnParams p) {
             cp_async16(sV + st * TILE_BYTES + d, vbase + off, ok ? 16 : 0);
         }
     };
+
+    // every stage of the ring is requested before anything else: a slice of a short context is then a
+    // single trip to memory, and the query loads below overlap with it
+#pragma unroll
+    for (int st = 0; st < kAttnStages; st++) {
+        if (st < nb) load_block(st);
+        cp_async_commit();
+    }
 
     // query fragments (A operand), scaled by log2(e)/sqrt(d_head) so that exp2 can be used.  Queries and
     // probabilities are carried as bf16 hi + bf16 lo (two MMAs each): a single bf16 rounding of q or p
@@ -136,16 +205,15 @@ k_attn_fd(const AttnParams p) {
     for (int n = 0; n < DH / 8; n++) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
-#pragma unroll
-    for (int st = 0; st < kAttnStages - 1; st++) {
-        if (st < nb) load_block(st);
-        cp_async_commit();
-    }
     for (int blk = 0; blk < nb; blk++) {
-        cp_async_wait<kAttnStages - 2>();
+        if (blk > 0) {
+            // everybody is done with block blk-1: its stage takes block blk-1+stages
+            __syncthreads();
+            if (blk - 1 + kAttnStages < nb) load_block(blk - 1 + kAttnStages);
+            cp_async_commit();
+        }
+        cp_async_wait<kAttnStages - 1>();
         __syncthreads();
-        if (blk + kAttnStages - 1 < nb) load_block(blk + kAttnStages - 1);
-        cp_async_commit();
         const int st = blk % kAttnStages;
         const uint32_t kS = sK + st * TILE_BYTES, vS = sV + st * TILE_BYTES;
 #pragma unroll
@@ -293,51 +361,11 @@ k_attn_fd(const AttnParams p) {
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    // The last slice merges all slices.  First the (max, sum) pairs of every slice and row go to
-    // shared memory as ready-made weights, then each output element needs one batch of independent
-    // loads: no load waits for a store.
+    // The last slice merges all slices.
     const size_t hb = (size_t)(b * p.md.H + head) * p.n_split * 32;
     float* sm_f = reinterpret_cast<float*>(smem_attn);             // [n_split][32] weight of slice s for row i
-    for (int i = tid; i < M; i += 128) {
-        float mm = -INFINITY;
-        for (int sidx = 0; sidx < p.n_split; sidx++) mm = fmaxf(mm, __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2));
-        float ll = 0.f;
-        for (int sidx = 0; sidx < p.n_split; sidx++) {
-            const float ms = __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2);
-            const float f = ms == -INFINITY ? 0.f : exp2f(ms - mm);
-            ll += __ldcg(p.part_ml + (hb + sidx * 32 + i) * 2 + 1) * f;
-            sm_f[sidx * 32 + i] = f;
-        }
-        const float inv = 1.f / ll;
-        for (int sidx = 0; sidx < p.n_split; sidx++) sm_f[sidx * 32 + i] *= inv;
-    }
-    __syncthreads();
-    constexpr int EB = 4;                                          // elements per thread and batch
-    for (int base = 0; base < M * DH; base += 128 * EB) {
-        float vals[EB][kAttnMaxSplit];
-#pragma unroll
-        for (int e = 0; e < EB; e++) {
-            const int idx = min(base + e * 128 + tid, M * DH - 1);
-            const int i = idx / DH, dcol = idx % DH;
-#pragma unroll
-            for (int sidx = 0; sidx < kAttnMaxSplit; sidx++)
-                vals[e][sidx] = sidx < p.n_split ? __ldcg(p.part_o + (hb + sidx * 32 + i) * DH + dcol) : 0.f;
-        }
-#pragma unroll
-        for (int e = 0; e < EB; e++) {
-            const int idx = base + e * 128 + tid;
-            if (idx < M * DH) {
-                const int i = idx / DH, dcol = idx % DH;
-                float v = 0.f;
-#pragma unroll
-                for (int sidx = 0; sidx < kAttnMaxSplit; sidx++)
-                    if (sidx < p.n_split) v += vals[e][sidx] * sm_f[sidx * 32 + i];
-                const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-                p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
-            }
-        }
-    }
+    if (p.n_split <= 4) attn_merge<DH, 4, 12>(p, hb, row0, head, sm_f);
+    else attn_merge<DH, kAttnMaxSplit, 4>(p, hb, row0, head, sm_f);
 }
 
 }  // namespace pass
