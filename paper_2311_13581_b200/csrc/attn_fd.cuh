@@ -35,6 +35,7 @@ struct AttnParams {
     int* counters;                 // [B*H], zero between launches
     __nv_bfloat16* out;            // [rows][d] hi parts, lo parts lo_row0 rows further down
     int lo_row0;
+    int debug_stale;               // test hook: the early part pretends the tables said len - debug_stale
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -131,25 +132,42 @@ k_attn_fd(const AttnParams p) {
     __shared__ int s_last;
 
     // Programmatic dependent launch: let the next kernel (the output projection) become resident and
-    // start streaming its weights now; this kernel's inputs come from the previous one, so wait for it.
+    // start streaming its weights now.  This kernel itself is resident long before its queries exist, and
+    // uses the time: blocks that hold nothing but cache rows of earlier steps (positions < len, which no
+    // kernel of this step writes) are fetched before the wait.  The row tables they are addressed through
+    // are read again after the wait; should they differ (this part ran before the tables of this step were
+    // written), everything is fetched again.  Rows of this step are written by the kernel being waited
+    // for and are touched only after the wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int head = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int mt = warp % MT, part = warp / MT;
     const int M = p.M, row0 = b * M;
-    const int seq = p.row_seq[row0], len = p.row_pos[row0];
-    const int n_tot = len + M;
-    // keys are dealt out in granules of 16 (one warp's share of a block), so that no slice is left
-    // empty while another holds a whole block more
-    int chunk = (n_tot + p.n_split - 1) / p.n_split;
-    chunk = ((chunk + 15) / 16) * 16;
-    const int k_begin = split * chunk;
-    const int k_end = min(n_tot, k_begin + chunk);
-    const int nb = k_end > k_begin ? (k_end - k_begin + kAttnBK - 1) / kAttnBK : 0;
-
-    const __nv_bfloat16* kbase = p.kc + kv_index(p.md, p.layer, seq, head, 0);
-    const __nv_bfloat16* vbase = p.vc + kv_index(p.md, p.layer, seq, head, 0);
+    // one thread reads the tables for all, so that the whole CTA works from the same pair even if it
+    // reads while they are being written
+    __shared__ int s_tab[2];
+    if (tid == 0) {
+        s_tab[0] = *(volatile const int*)(p.row_seq + row0);
+        s_tab[1] = *(volatile const int*)(p.row_pos + row0);
+    }
+    __syncthreads();
+    int seq, len, k_begin, k_end, nb;
+    const __nv_bfloat16 *kbase, *vbase;
+    auto slice = [&](int seq_, int len_) {
+        seq = seq_;
+        len = len_;
+        const int n_tot = len + M;
+        // keys are dealt out in granules of 16 (one warp's share of a block), so that no slice is left
+        // empty while another holds a whole block more
+        int chunk = (n_tot + p.n_split - 1) / p.n_split;
+        chunk = ((chunk + 15) / 16) * 16;
+        k_begin = split * chunk;
+        k_end = min(n_tot, k_begin + chunk);
+        nb = k_end > k_begin ? (k_end - k_begin + kAttnBK - 1) / kAttnBK : 0;
+        kbase = p.kc + kv_index(p.md, p.layer, seq, head, 0);
+        vbase = p.vc + kv_index(p.md, p.layer, seq, head, 0);
+    };
+    slice(s_tab[0], max(0, s_tab[1] - p.debug_stale));
     const uint32_t sK = smem_u32(smem_attn), sV = sK + kAttnStages * TILE_BYTES;
 
     auto load_block = [&](int blk) {
@@ -166,11 +184,27 @@ k_attn_fd(const AttnParams p) {
         }
     };
 
-    // every stage of the ring is requested before anything else: a slice of a short context is then a
-    // single trip to memory, and the query loads below overlap with it
+    // first ring fill: blocks of old rows now, the rest (and the queries) after the wait
+    uint32_t early = 0;
 #pragma unroll
     for (int st = 0; st < kAttnStages; st++) {
-        if (st < nb) load_block(st);
+        if (st < nb && min(k_end, k_begin + (st + 1) * kAttnBK) <= len) { load_block(st); early |= 1u << st; }
+    }
+    cp_async_commit();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    {
+        const int seq_f = __ldcg(p.row_seq + row0), len_f = __ldcg(p.row_pos + row0);    // final now, the same for every thread
+        if (seq_f != seq || len_f != len) {
+            // the early part worked from tables of an earlier step: let its copies land, then start over
+            cp_async_wait<0>();
+            __syncthreads();
+            slice(seq_f, len_f);
+            early = 0;
+        }
+    }
+#pragma unroll
+    for (int st = 0; st < kAttnStages; st++) {
+        if (st < nb && !((early >> st) & 1u)) load_block(st);
         cp_async_commit();
     }
 

@@ -134,6 +134,7 @@ struct pass_ctx {
     int* d_attn_cnt = nullptr;
     int n_sms = 148;
     bool use_pdl = true;
+    int attn_debug_stale = 0;     // PASS_ATTN_STALE=n: attention's early part works from a cache length n short
     bool use_tc = false;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
     int trace_launch = 0;
@@ -476,7 +477,7 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
-            ap.out = c->d_attn_bf; ap.lo_row0 = rh;
+            ap.out = c->d_attn_bf; ap.lo_row0 = rh; ap.debug_stale = c->attn_debug_stale;
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
             else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
         } else if (md.dh == 128) {
@@ -650,6 +651,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_chain_flags = (int*)(w + L.chain_flags);
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
+        if (const char* e = getenv("PASS_ATTN_STALE")) c->attn_debug_stale = std::max(0, atoi(e));
         c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) == cudaSuccess &&

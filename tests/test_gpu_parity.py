@@ -227,6 +227,22 @@ def test_tiny_bf16_long_prompt_many_key_blocks(k):
     ctx.close()
 
 
+def test_attention_restarts_when_its_early_fetch_used_outdated_row_tables(monkeypatch):
+    """The attention kernel fetches old cache rows before its queries exist, from row tables it reads
+    ahead of the kernel it depends on, and starts over if those turn out to be outdated.  On a normal
+    run they never are, so the hook makes the early part work from a cache length 70 short (another
+    split of the keys, other blocks in the ring): results must not change."""
+    from parity_util import lockstep, make_pair
+    monkeypatch.setenv("PASS_ATTN_STALE", "70")
+    prompt = si.make_prompt(TINY_BF16, 333)
+    ctx, oracles, _ = make_pair(TINY_BF16, 1, 333 + 80, [prompt], seed=1)
+    stats, _ = lockstep(ctx, oracles, 4, 0.8, 4, check_A=False)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    stats, _ = lockstep(ctx, oracles, 4, 0.0, 3, step0=4, check_A=True)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
 def _load_synthetic_cache(ctx, oracle_backends, shape, n_pos, std=1.0):
     for b, be in enumerate(oracle_backends):
         for layer in range(shape.n_layers):
