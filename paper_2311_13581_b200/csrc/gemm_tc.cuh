@@ -385,7 +385,9 @@ struct ChainParams {
     int n_ops;
     int stages;
     int npad;                  // row padding, shared by all GEMMs of the chain
-    int pf_units;              // how far beyond the ring weights are pulled into L2 while the ring is stalled
+    int pf_units;              // stages per GEMM that are pulled into L2 while the CTA waits for the previous GEMM
+    int hold;                  // experiment: no weight request for a GEMM before this CTA's epilogue of the previous one is over
+    int pf_units0;             // the same for the first GEMM of the launch (waits for the previous kernel)
     int* op_done;              // [kMaxOps] tiles completed per GEMM; zero between launches
     int* ctas_done;            // CTAs that have left the kernel (the last one clears op_done)
     int* status;
@@ -435,6 +437,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ int s_issued, s_issued_b;
+    __shared__ int s_epi_done;
+    __shared__ int s_mma_done;             // last GEMM of the chain whose MMAs this CTA has all issued (-1: none)
     __shared__ int s_last;
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
@@ -478,6 +482,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         s_abort = 0;
         s_issued = 0;
         s_issued_b = 0;
+        s_mma_done = -1;
+        s_epi_done = -1;
         s_epi_fail = 0;
         fence_barrier_init();
     }
@@ -505,6 +511,13 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
                 const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
+                if (cp.hold && oi > 0) {
+                    const long long t0 = clock64();
+                    while (*(volatile int*)&s_epi_done < oi - 1) {
+                        if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { ok = false; break; }
+                        __nanosleep(100);
+                    }
+                }
                 for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
@@ -565,12 +578,19 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         // rows with prefetch.global.L2: one 128-byte row segment per lane and instruction.  These go
         // through the load/store path, not through the TMA queue, so they never sit in front of the
         // ring's own requests; they keep HBM streaming while the consumers wait for an earlier GEMM.
-        if (cp.pf_units > 0) {
+        if (cp.pf_units > 0 || cp.pf_units0 > 0) {
+            // One burst per GEMM: when this CTA has issued the last MMA of the previous GEMM, its ring
+            // already holds the first stages of the next one and nothing more can be requested until the
+            // previous GEMM's results exist everywhere.  HBM would idle through that hand-over; instead
+            // the stages that follow the ring's are pulled into L2 now.  Nothing is prefetched while
+            // the previous GEMM still streams (that would only delay the data it is waiting for).
             int count = 0;
             Piece pc;
             bool stop = false;
             for (int oi = 0; !stop && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
+                const int burst = oi == 0 ? cp.pf_units0 : cp.pf_units;
+                int in_op = 0;
                 for (int it = 0; !stop && fetch_piece(oi, it, pc); it++) {
                     // rows of the tile: plain = 128 rows of one matrix; interleaved = 64 rows of two
                     const char* base0; const char* base1; int row0, nrows0, nrows1;
@@ -584,15 +604,15 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         row0 = tl * kTileN; nrows0 = min(kTileN, p.w_rows[seg] - row0); nrows1 = 0;
                     }
                     const size_t ldb = (size_t)p.w_ld * 2;
-                    for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++) {
+                    for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++, in_op++) {
+                        if (in_op < S || in_op >= S + burst) continue;      // the ring's own / beyond the burst
                         const long long t0 = clock64();
-                        int issued;
-                        while (count >= (issued = *(volatile int*)&s_issued) + S + cp.pf_units) {
+                        while (*(volatile int*)&s_mma_done < oi - 1) {
                             if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { stop = true; break; }
-                            __nanosleep(100);
+                            __nanosleep(200);
                         }
                         if (stop) break;
-                        if (count < issued + S) continue;                   // the ring got there first
+                        if (count < *(volatile int*)&s_issued) continue;    // the ring got there first
                         const size_t col = (size_t)kb * kBlockK * 2;
                         if ((kb + 1) * kBlockK > p.w_ld) continue;          // ragged last k-block: leave it to TMA
                         for (int r = lane; r < nrows0; r += 32)
@@ -633,6 +653,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     }
                     if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
                 }
+                *(volatile int*)&s_mma_done = oi;
                 PASS_TRACE(oi, 2);
             }
         }
@@ -708,10 +729,11 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     if (whole) {
                         epi_store(p, ec, pc.tile, c0, hi);
                     } else {
-                        // partial slot layout [feature][rh]: each thread owns 4*rh contiguous bytes
-                        float4* dst = reinterpret_cast<float4*>(my_slot + (size_t)ec.lane_in_tile * p.rh + c0);
+                        // partial slot layout [rh/4][feature] of float4 (four token rows of one feature): a warp
+                        // stores and loads 512 contiguous bytes per instruction
+                        float4* dst = reinterpret_cast<float4*>(my_slot) + (size_t)(c0 >> 2) * kTileN + ec.lane_in_tile;
                         dst[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                        dst[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
+                        dst[kTileN] = make_float4(hi[4], hi[5], hi[6], hi[7]);
                     }
                 }
                 tc_fence_before();
@@ -764,10 +786,10 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                     const int cq = c_first + qi;
                                     const int slot = qi == 0 ? slot_first : 0;
                                     const float4* src = reinterpret_cast<const float4*>(
-                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * 16);
+                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats) + ec.lane_in_tile;
 #pragma unroll
                                     for (int f = 0; f < 4; f++)
-                                        v[qq][f] = (f < nf4 && q0 + qq < pc.n_pieces) ? __ldcg(src + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                        v[qq][f] = (f < nf4 && q0 + qq < pc.n_pieces) ? __ldcg(src + f * kTileN) : make_float4(0.f, 0.f, 0.f, 0.f);
                                 }
 #pragma unroll
                                 for (int qq = 0; qq < 6; qq++) {
@@ -777,6 +799,13 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                         acc[f >> 1][(f & 1) * 4 + 2] += v[qq][f].z; acc[f >> 1][(f & 1) * 4 + 3] += v[qq][f].w;
                                     }
                                 }
+                            }
+                            if (cp.hold == 2) {
+                                // the loads are over: weights of the next GEMM may be requested
+                                const int dep = __any_sync(0xffffffffu, acc[0][0] + acc[1][7] == 1.2345e30f);
+                                bool more = false;
+                                { Piece nx; more = fetch_piece(oi, it + 1, nx); }
+                                if (et == 0 && !more) *(volatile int*)&s_epi_done = oi + dep;
                             }
                             epi_store(p, ec, pc.tile, 0, acc[0], p.epi == kEpiResid ? hv[0] : nullptr,
                                       p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs_pre : nullptr);
@@ -798,9 +827,9 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                     // every contributor but the first starts its own range inside this tile
                                     const int slot = qi == 0 ? slot_first : 0;
                                     const float4* src = reinterpret_cast<const float4*>(
-                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats + (size_t)ec.lane_in_tile * p.rh + c0);
+                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats) + (size_t)(c0 >> 2) * kTileN + ec.lane_in_tile;
                                     v[qq][0] = __ldcg(src);
-                                    v[qq][1] = __ldcg(src + 1);
+                                    v[qq][1] = __ldcg(src + kTileN);
                                 }
 #pragma unroll
                                 for (int qq = 0; qq < 8; qq++) {
@@ -823,6 +852,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     if (et == 0) PASS_TRACE(oi, 7);
                 }
             }
+            if (et == 0) *(volatile int*)&s_epi_done = oi;
             if (et == 0) PASS_TRACE(oi, 3);
         }
     }
