@@ -386,7 +386,8 @@ struct ChainParams {
     int stages;
     int npad;                  // row padding, shared by all GEMMs of the chain
     int pf_units;              // stages per GEMM that are pulled into L2 while the CTA waits for the previous GEMM
-    int hold;                  // experiment: no weight request for a GEMM before this CTA's epilogue of the previous one is over
+    int hold;                  // 1: no weight request for a GEMM before this CTA's epilogue of the previous one is over
+                               // (measured: the hand-over's own trips to L2 are shorter when the ring is not refilling)
     int pf_units0;             // the same for the first GEMM of the launch (waits for the previous kernel)
     int* op_done;              // [kMaxOps] tiles completed per GEMM; zero between launches
     int* ctas_done;            // CTAs that have left the kernel (the last one clears op_done)
@@ -698,7 +699,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 // what the epilogue of this tile reads besides the accumulator is requested now, so that
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
-                float2 cs_pre[16];
+                float2 cs_pre[16] = {};
                 const bool pre = p.rh == 16 && pc.n_pieces > 1;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
@@ -766,7 +767,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                             // values and the parts of four contributors are requested together, so the whole
                             // reduction costs one or two trips to L2 instead of one per half and contributor group.
                             const int n = pc.tile * kTileN + ec.lane_in_tile;
-                            float hv[2][8];
+                            float hv[2][8] = {};
                             if (p.epi == kEpiResid) {
 #pragma unroll
                                 for (int j = 0; j < 16; j++)
@@ -800,17 +801,23 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                     }
                                 }
                             }
-                            if (cp.hold == 2) {
-                                // the loads are over: weights of the next GEMM may be requested
-                                const int dep = __any_sync(0xffffffffu, acc[0][0] + acc[1][7] == 1.2345e30f);
-                                bool more = false;
-                                { Piece nx; more = fetch_piece(oi, it + 1, nx); }
-                                if (et == 0 && !more) *(volatile int*)&s_epi_done = oi + dep;
+                            // both halves run through ONE copy of the epilogue code (the loop is kept rolled):
+                            // this code runs once per GEMM and CTA, so every instruction line of it is a
+                            // fetch from L2, and a second inlined copy would pay for its lines again
+#pragma unroll 1
+                            for (int half = 0; half < 2; half++) {
+                                if (half * 8 >= p.R) break;
+                                float a8[8], h8[8];
+                                float2 cs8[8];
+#pragma unroll
+                                for (int j = 0; j < 8; j++) {
+                                    a8[j] = half ? acc[1][j] : acc[0][j];
+                                    h8[j] = half ? hv[1][j] : hv[0][j];
+                                    cs8[j] = half ? cs_pre[8 + j] : cs_pre[j];
+                                }
+                                epi_store(p, ec, pc.tile, half * 8, a8, p.epi == kEpiResid ? h8 : nullptr,
+                                          p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs8 : nullptr);
                             }
-                            epi_store(p, ec, pc.tile, 0, acc[0], p.epi == kEpiResid ? hv[0] : nullptr,
-                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs_pre : nullptr);
-                            epi_store(p, ec, pc.tile, 8, acc[1], p.epi == kEpiResid ? hv[1] : nullptr,
-                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs_pre + 8 : nullptr);
                         } else
                         for (int c0 = 0; c0 < p.rh; c0 += 8) {
                             float acc[8];
