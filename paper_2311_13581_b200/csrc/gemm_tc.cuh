@@ -224,26 +224,53 @@ __device__ __forceinline__ int unit_owner(long long x, long long U, long long G)
 }
 
 // The it-th piece of CTA `c`; returns false when the CTA's range is exhausted.
+//
+// With at least as many tiles as CTAs the schedule has two phases.  First the n_tiles mod G "odd" tiles
+// are streamed: their (tile, k-block) units are dealt out evenly, so tiles are shared and the last CTA to
+// deliver sums the parts - early in the GEMM, while the MMAs already work on what follows.  Then every
+// CTA computes whole tiles of its own.  The GEMM therefore ends on whole tiles, whose epilogue needs no
+// other CTA: no arrival counter and no trip for partial sums on the path to the next GEMM.  With fewer
+// tiles than CTAs everything is streamed.
 __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
-    const long long U = (long long)p.n_tiles * p.kb_per_tile;
-    if (G > U) G = (int)U;            // fewer units than CTAs: only the first U CTAs work on this GEMM
-    if (c >= G) return false;
-    const long long s = unit_start(c, U, G), e = unit_start(c + 1, U, G);
-    if (s >= e) return false;
-    const int t0 = (int)(s / p.kb_per_tile);
-    const int tile = t0 + it;
-    const long long ts = (long long)tile * p.kb_per_tile;
-    if (ts >= e) return false;
-    const long long a = ts > s ? ts : s;
-    const long long b = (ts + p.kb_per_tile) < e ? (ts + p.kb_per_tile) : e;
-    out.tile = tile;
-    out.kb0 = (int)(a - ts);
-    out.kb1 = (int)(b - ts);
-    const int c_first = unit_owner(ts, U, G), c_last = unit_owner(ts + p.kb_per_tile - 1, U, G);
-    out.n_pieces = c_last - c_first + 1;
-    out.index = c - c_first;
-    out.slot = (a == s) ? 0 : 1;
-    out.first_slot = (unit_start(c_first, U, G) >= ts) ? 0 : 1;
+    const int rounds = p.n_tiles >= G ? p.n_tiles / G : 0;      // whole tiles per CTA
+    const int n_sk = p.n_tiles - rounds * G;                     // tiles that are streamed, [0, n_sk)
+    const long long U = (long long)n_sk * p.kb_per_tile;
+    int sk_pieces = 0;
+    if (U > 0) {
+        int Gs = G;
+        if (Gs > U) Gs = (int)U;      // fewer units than CTAs: only the first U CTAs stream
+        if (c < Gs) {
+            const long long s = unit_start(c, U, Gs), e = unit_start(c + 1, U, Gs);
+            if (s < e) {
+                const int t0 = (int)(s / p.kb_per_tile);
+                sk_pieces = (int)((e - 1) / p.kb_per_tile) - t0 + 1;
+                if (it < sk_pieces) {
+                    const int tile = t0 + it;
+                    const long long ts = (long long)tile * p.kb_per_tile;
+                    const long long a = ts > s ? ts : s;
+                    const long long b = (ts + p.kb_per_tile) < e ? (ts + p.kb_per_tile) : e;
+                    out.tile = tile;
+                    out.kb0 = (int)(a - ts);
+                    out.kb1 = (int)(b - ts);
+                    const int c_first = unit_owner(ts, U, Gs), c_last = unit_owner(ts + p.kb_per_tile - 1, U, Gs);
+                    out.n_pieces = c_last - c_first + 1;
+                    out.index = c - c_first;
+                    out.slot = (a == s) ? 0 : 1;
+                    out.first_slot = (unit_start(c_first, U, Gs) >= ts) ? 0 : 1;
+                    return true;
+                }
+            }
+        }
+    }
+    const int j = it - sk_pieces;
+    if (j >= rounds) return false;
+    out.tile = n_sk + j * G + c;
+    out.kb0 = 0;
+    out.kb1 = p.kb_per_tile;
+    out.n_pieces = 1;
+    out.index = 0;
+    out.slot = 0;
+    out.first_slot = 0;
     return true;
 }
 
@@ -681,15 +708,30 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 epi_bar();
                 if (*(volatile int*)&s_epi_fail) { ok = false; break; }
             }
-            for (int r = et; r < p.R; r += 128) {
-                float rs = 1.f;
-                if (p.sumsq_in) {
-                    float ss = 0.f;
-                    for (int t = 0; t < p.n_parts_in; t++) ss += __ldcg(p.sumsq_in + (size_t)t * kMaxRows + r);
-                    rs = rsqrtf(ss * p.inv_d_in + p.eps);
+            // rstd of the input rows: eight lanes per row, each sums every eighth part (its loads are
+            // independent, so a row costs one trip to L2 whatever the number of parts), then a fixed-order
+            // butterfly.  The first accumulator of a short first piece may already be waiting for us.
+            for (int r0 = 0; r0 < p.R; r0 += 16) {
+                const int r = r0 + (et >> 3), l8 = et & 7;
+                float ss = 0.f;
+                if (p.sumsq_in && r < p.R) {
+                    float part[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int t0 = 0; t0 < p.n_parts_in; t0 += 32) {
+#pragma unroll
+                        for (int u = 0; u < 4; u++) {
+                            const int t = t0 + u * 8 + l8;
+                            if (t < p.n_parts_in) part[u] += __ldcg(p.sumsq_in + (size_t)t * kMaxRows + r);
+                        }
+                    }
+                    ss = (part[0] + part[1]) + (part[2] + part[3]);
                 }
-                s_rstd[r] = rs;
-                if (p.epi == kEpiQKV) { s_rseq[r] = __ldg(p.row_seq + r); s_rpos[r] = __ldg(p.row_pos + r); }
+                ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+                if (r < p.R && l8 == 0) {
+                    s_rstd[r] = p.sumsq_in ? rsqrtf(ss * p.inv_d_in + p.eps) : 1.f;
+                    if (p.epi == kEpiQKV) { s_rseq[r] = __ldg(p.row_seq + r); s_rpos[r] = __ldg(p.row_pos + r); }
+                }
             }
             epi_bar();
             const size_t slot_floats = (size_t)p.rh * kTileN;
@@ -757,9 +799,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     if (et == 0) PASS_TRACE(oi, 5);
                     if (s_last) {
                         tile_done = true;
-                        const long long U = (long long)p.n_tiles * p.kb_per_tile;
-                        const long long ts = (long long)pc.tile * p.kb_per_tile;
-                        const int Ge = G > U ? (int)U : G;
                         const int c_first = cta - pc.index;
                         const int slot_first = pc.first_slot;
                         if (p.rh == 16) {
