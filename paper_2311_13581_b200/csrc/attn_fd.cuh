@@ -122,7 +122,25 @@ __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int r
     }
 }
 
-template <int DH, int MT>
+// CL: the slices of one (sequence, head) form a thread-block cluster (n_split CTAs along z) and are
+// merged through distributed shared memory: every CTA leaves its slice's unnormalised output and its
+// (max, sum) pairs in its own shared memory, the cluster synchronises once, and each CTA then merges a
+// share of the output rows reading all slices with ld.shared::cluster.  Compared with the merge through
+// global memory this saves the partial stores, the fence, the arrival counter and a trip to L2.
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t ra;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+template <int DH, int MT, bool CL>
 __global__ void __launch_bounds__(128)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
@@ -378,12 +396,53 @@ k_attn_fd(const AttnParams p) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
             p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
             p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        } else if (CL) {
+            float* cl_o = sm_o + 4 * 16 * DH + 128;          // [32][DH], behind the warp staging area
+            float* cl_ml = cl_o + 32 * DH;                   // [32][2]
+            cl_o[i * DH + dcol] = acc;
+            if (dcol == 0) { cl_ml[i * 2] = mm; cl_ml[i * 2 + 1] = ll; }
         } else {
             p.part_o[(pbase + i) * DH + dcol] = acc;
             if (dcol == 0) { p.part_ml[(pbase + i) * 2] = mm; p.part_ml[(pbase + i) * 2 + 1] = ll; }
         }
     }
     if (p.n_split == 1) return;
+    if (CL) {
+        constexpr int NSMAX = 8;
+        const uint32_t cl_o_addr = smem_u32(sm_o + 4 * 16 * DH + 128), cl_ml_addr = cl_o_addr + 32 * DH * 4;
+        const int ns = p.n_split;
+        const uint32_t rank = cluster_ctarank();
+        cluster_sync_all();                                  // every slice's partials are in place
+        for (int idx = (int)rank * 128 + tid; idx < M * DH; idx += ns * 128) {
+            const int i = idx / DH;
+            float ms[NSMAX], ls[NSMAX], os[NSMAX];
+#pragma unroll
+            for (int sidx = 0; sidx < NSMAX; sidx++) {
+                if (sidx < ns) {
+                    ms[sidx] = ld_dsmem_f32(cl_ml_addr + (uint32_t)(i * 2) * 4, sidx);
+                    ls[sidx] = ld_dsmem_f32(cl_ml_addr + (uint32_t)(i * 2 + 1) * 4, sidx);
+                    os[sidx] = ld_dsmem_f32(cl_o_addr + (uint32_t)idx * 4, sidx);
+                } else { ms[sidx] = -INFINITY; ls[sidx] = 0.f; os[sidx] = 0.f; }
+            }
+            float mm = -INFINITY;
+#pragma unroll
+            for (int sidx = 0; sidx < NSMAX; sidx++) mm = fmaxf(mm, ms[sidx]);
+            float ll = 0.f, v = 0.f;
+#pragma unroll
+            for (int sidx = 0; sidx < NSMAX; sidx++) {
+                const float f = ms[sidx] == -INFINITY ? 0.f : exp2f(ms[sidx] - mm);
+                ll += ls[sidx] * f;
+                v += os[sidx] * f;
+            }
+            v /= ll;
+            const int dcol = idx % DH;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
+            p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        }
+        cluster_sync_all();                                  // nobody leaves while its memory is still being read
+        return;
+    }
 
     __threadfence();
     __syncthreads();

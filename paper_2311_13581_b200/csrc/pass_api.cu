@@ -134,6 +134,7 @@ struct pass_ctx {
     int* d_attn_cnt = nullptr;
     int n_sms = 148;
     bool use_pdl = true;
+    bool attn_cluster = true;     // PASS_ATTN_NO_CLUSTER: merge attention slices through global memory
     int attn_debug_stale = 0;     // PASS_ATTN_STALE=n: attention's early part works from a cache length n short
     bool use_tc = false;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
@@ -364,13 +365,13 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
 
 // The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
 // attention, O GEMM (+residual, next norm's input), gate/up GEMM (+SwiGLU), down GEMM (+residual).
-template <int DH, int MT>
-static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
+template <int DH, int MT, bool CL>
+static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
     static bool set = false;
     if (!set) {
-        cudaFuncSetAttribute(k_attn_fd<DH, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        cudaFuncSetAttribute(k_attn_fd<DH, MT>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
         set = true;
     }
     cudaLaunchConfig_t cfg;
@@ -379,13 +380,55 @@ static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
     cfg.blockDim = dim3(128);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = c->stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (CL) {
+        at[na].id = cudaLaunchAttributeClusterDimension;
+        at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = ap.n_split;
+        na++;
+    }
+    if (c->use_pdl) {
+        at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[na].val.programmaticStreamSerializationAllowed = 1;
+        na++;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = c->use_pdl ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT>, ap);
+    cfg.numAttrs = na;
+    cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL>, ap);
     c->launches++;
+}
+
+// Can the slices of every (sequence, head) run as one cluster each, all at the same time?  Asked once per
+// kernel instance and slice count; if not (or with more than 8 slices) the merge goes through global memory.
+template <int DH, int MT>
+static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
+    if (!c->attn_cluster || n_split < 2 || n_split > 8) return false;
+    static int cached_split = -1, cached_max = 0;
+    if (cached_split != n_split) {
+        constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
+        cudaFuncSetAttribute(k_attn_fd<DH, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(c->md.H, n_seq, n_split);
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = n_split;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        cached_split = n_split;
+        cached_max = n;
+    }
+    return cached_max >= c->md.H * n_seq;
+}
+
+template <int DH, int MT>
+static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
+    if (attn_cluster_ok<DH, MT>(c, ap.n_split, n_seq)) launch_attn_fd_impl<DH, MT, true>(c, ap, n_seq);
+    else launch_attn_fd_impl<DH, MT, false>(c, ap, n_seq);
 }
 
 // GEMMs of the decoder layers as chain entries.
@@ -654,6 +697,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_chain_flags = (int*)(w + L.chain_flags);
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
+        c->attn_cluster = getenv("PASS_ATTN_NO_CLUSTER") == nullptr;
         if (const char* e = getenv("PASS_ATTN_STALE")) c->attn_debug_stale = std::max(0, atoi(e));
         c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
