@@ -140,8 +140,9 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
     return v;
 }
 
+// 168 registers x 128 threads is what is left on an SM beside the GEMM kernel's CTA (256 x 168).
 template <int DH, int MT, bool CL>
-__global__ void __launch_bounds__(128)
+__global__ void __maxnreg__(168)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
     constexpr int CH = DH / 8;                       // 16-byte chunks per key
@@ -273,9 +274,9 @@ k_attn_fd(const AttnParams p) {
             const int key0 = part * KPW + sub * 16;          // within the block
             const int gkey0 = k_begin + blk * kAttnBK + key0;
             if (gkey0 >= k_end) continue;
-            float s[2][4];
+            float s[2][4], sl[2][4];      // hi and lo query parts accumulate apart: four chains of 8 MMAs, not two of 16
 #pragma unroll
-            for (int n = 0; n < 2; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+            for (int n = 0; n < 2; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; sl[n][0] = sl[n][1] = sl[n][2] = sl[n][3] = 0.f; }
             {
                 const int mi = lane >> 3, rr = lane & 7;
                 const int key = key0 + (mi >> 1) * 8 + rr;
@@ -286,9 +287,13 @@ k_attn_fd(const AttnParams p) {
                     ldsm_x4(kS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
                     mma_bf16_16816(s[0], qf[ks], r[0], r[1]);
                     mma_bf16_16816(s[1], qf[ks], r[2], r[3]);
-                    mma_bf16_16816(s[0], qfl[ks], r[0], r[1]);
-                    mma_bf16_16816(s[1], qfl[ks], r[2], r[3]);
+                    mma_bf16_16816(sl[0], qfl[ks], r[0], r[1]);
+                    mma_bf16_16816(sl[1], qfl[ks], r[2], r[3]);
                 }
+#pragma unroll
+                for (int n = 0; n < 2; n++)
+#pragma unroll
+                    for (int e = 0; e < 4; e++) s[n][e] += sl[n][e];
             }
             // causal mask: row i sees key j iff j <= len + i
             const int i0 = mt * 16 + g, i1 = i0 + 8;
@@ -364,10 +369,17 @@ k_attn_fd(const AttnParams p) {
     float* sm_o = reinterpret_cast<float*>(smem_attn);
     float* sm_m = sm_o + 4 * 16 * DH;
     float* sm_l = sm_m + 64;
+    // staging rows are swizzled in blocks of 8 floats by (row & 3) so that the eight rows a warp writes
+    // at once fall into different banks; rows beyond M are not written (nobody reads them)
+    {
+        const bool live0 = mt * 16 + g < M, live1 = mt * 16 + g + 8 < M;
+        const int sw = (g & 3) * 8;
 #pragma unroll
-    for (int n = 0; n < DH / 8; n++) {
-        *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g) * DH + n * 8 + 2 * t)) = make_float2(o[n][0], o[n][1]);
-        *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g + 8) * DH + n * 8 + 2 * t)) = make_float2(o[n][2], o[n][3]);
+        for (int n = 0; n < DH / 8; n++) {
+            const int col = (n * 8 + 2 * t) ^ sw;
+            if (live0) *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g) * DH + col)) = make_float2(o[n][0], o[n][1]);
+            if (live1) *reinterpret_cast<float2*>(sm_o + ((warp * 16 + g + 8) * DH + col)) = make_float2(o[n][2], o[n][3]);
+        }
     }
     if (t == 0) {
         sm_m[warp * 16 + g] = m_run[0]; sm_m[warp * 16 + g + 8] = m_run[1];
@@ -388,7 +400,7 @@ k_attn_fd(const AttnParams p) {
             const int w = q * MT + tile;
             const float mw = sm_m[w * 16 + rr];
             const float f = mw == -INFINITY ? 0.f : exp2f(mw - mm);
-            acc += sm_o[(w * 16 + rr) * DH + dcol] * f;
+            acc += sm_o[(w * 16 + rr) * DH + (dcol ^ ((rr & 3) * 8))] * f;
             ll += sm_l[w * 16 + rr] * f;
         }
         if (p.n_split == 1) {
