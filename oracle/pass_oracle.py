@@ -257,8 +257,21 @@ class TableBackend:
 # Sampling primitives
 # ---------------------------------------------------------------------------
 
-def softmax_T(z: np.ndarray, temperature: float) -> np.ndarray:
-    """softmax(z / T) in float64; T == 0 is the one-hot law at the first argmax."""
+def top_k_set(z: np.ndarray, top_k: int) -> np.ndarray:
+    """Indices of the top_k largest entries of z; among equal values the lower index ranks first."""
+    z = np.asarray(z, dtype=np.float64)
+    order = sorted(range(z.size), key=lambda i: (-z[i], i))
+    return np.array(sorted(order[:top_k]), dtype=np.int64)
+
+
+def softmax_T(z: np.ndarray, temperature: float, top_k: int = 0) -> np.ndarray:
+    """softmax(z / T) in float64; T == 0 is the one-hot law at the first argmax.
+
+    top_k > 0 is top-k sampling (Experiments, setup: "top-k sampling" with a
+    temperature): the law is the softmax over the top_k largest logits only,
+    every other token has probability exactly 0.  The same filter is applied to
+    every row, target rows and look-ahead rows alike, before any ratio is formed.
+    """
     z = np.asarray(z, dtype=np.float64)
     if temperature == 0.0:
         p = np.zeros_like(z)
@@ -266,6 +279,10 @@ def softmax_T(z: np.ndarray, temperature: float) -> np.ndarray:
         return p
     s = z / float(temperature)
     e = np.exp(s - np.max(s))
+    if 0 < top_k < z.size:
+        keep = np.zeros(z.size, dtype=bool)
+        keep[top_k_set(z, top_k)] = True
+        e = np.where(keep, e, 0.0)
     return e / np.sum(e)
 
 
@@ -349,6 +366,8 @@ class PassOracle:
         self.Q_dft = np.zeros((0, backend.vocab))
         self.k_prev: Optional[int] = None
         self.T_prev: Optional[float] = None
+        self.top_k = 0                      # 0 = plain temperature sampling
+        self.top_k_prev = 0
         self.last_logits: Optional[np.ndarray] = None
 
     def rows(self, k: int) -> List[Row]:
@@ -357,9 +376,10 @@ class PassOracle:
 
     def forward_step(self, k: int, temperature: float) -> np.ndarray:
         """Run the model call of a step; returns float64 logits [1 + m + k, V]."""
-        if k != self.k_prev or temperature != self.T_prev:
+        top_k = getattr(self, "top_k", 0)
+        if k != self.k_prev or temperature != self.T_prev or top_k != getattr(self, "top_k_prev", 0):
             self.drafts, self.Q_dft = [], np.zeros((0, self.be.vocab))   # drawn under other settings
-        self.k_prev, self.T_prev = k, temperature
+        self.k_prev, self.T_prev, self.top_k_prev = k, temperature, top_k
         Z = self.be.forward(self.rows(k), self.len)
         self.last_logits = Z
         return Z
@@ -372,8 +392,9 @@ class PassOracle:
         other implementation computed.
         """
         m = len(self.drafts)
+        top_k = getattr(self, "top_k", 0)
         Z = np.asarray(Z, dtype=np.float64)
-        P_tgt = np.stack([softmax_T(Z[j], temperature) for j in range(m + 1)])
+        P_tgt = np.stack([softmax_T(Z[j], temperature, top_k) for j in range(m + 1)])
         a, y, info = verify(P_tgt, Q_dft, self.drafts, u[:m], u[k])
         info["final_margin"] = invcdf_margin(info["final_law"], u[k])
         srt = np.sort(Z[a])
@@ -382,7 +403,7 @@ class PassOracle:
         dec = {"m": m, "n_accepted": a, "final": y, "emitted": list(self.drafts[:a]) + [y],
                "new_drafts": [], "Qn": np.zeros((0, self.be.vocab)), "info": info}
         if a == m and k > 0:
-            Qn = np.stack([softmax_T(Z[m + 1 + t], temperature) for t in range(k)])
+            Qn = np.stack([softmax_T(Z[m + 1 + t], temperature, top_k) for t in range(k)])
             dec["Qn"] = Qn
             dec["new_drafts"] = [invcdf(Qn[t], u[k + 1 + t]) for t in range(k)]
             info["draft_margin"] = [invcdf_margin(Qn[t], u[k + 1 + t]) for t in range(k)]
@@ -398,8 +419,10 @@ class PassOracle:
         self.Q_dft = np.asarray(Qn, dtype=np.float64) if len(new_drafts) else \
             np.zeros((0, self.be.vocab))
 
-    def step(self, k: int, temperature: float, u: Sequence[float]):
+    def step(self, k: int, temperature: float, u: Sequence[float], top_k: Optional[int] = None):
         """Returns (emitted tokens, n_accepted, info).  1 <= len(emitted) <= k+1."""
+        if top_k is not None:
+            self.top_k = int(top_k)
         Z = self.forward_step(k, temperature)
         dec = self.decide(Z, self.Q_dft, k, temperature, u)
         self.commit(dec["emitted"], dec["new_drafts"], dec["Qn"])
@@ -407,7 +430,7 @@ class PassOracle:
 
 
 def alg1_two_call(backend, prompt: Sequence[int], L: int, temperature: float,
-                  n_tokens: int, uniform_fn: Callable[[int, int], np.ndarray]):
+                  n_tokens: int, uniform_fn: Callable[[int, int], np.ndarray], top_k: int = 0):
     """Algorithm 1 as printed: per iteration a drafting call on
     [x_n, LA_1..LA_L], then a validation call on [x_{n+1}, d_1..d_L].
 
@@ -426,8 +449,8 @@ def alg1_two_call(backend, prompt: Sequence[int], L: int, temperature: float,
         # drafting phase
         Z = backend.forward([("tok", pending)] + [("la", i) for i in range(L)], n_cached)
         calls += 1
-        x_next = invcdf(softmax_T(Z[0], temperature), u[0])
-        Q_dft = np.stack([softmax_T(Z[1 + t], temperature) for t in range(L)])
+        x_next = invcdf(softmax_T(Z[0], temperature, top_k), u[0])
+        Q_dft = np.stack([softmax_T(Z[1 + t], temperature, top_k) for t in range(L)])
         drafts = [invcdf(Q_dft[t], u[1 + t]) for t in range(L)]
         out.append(x_next)
         n_cached += 1                      # keep K/V of the old pending token only
@@ -435,7 +458,7 @@ def alg1_two_call(backend, prompt: Sequence[int], L: int, temperature: float,
         # validation phase
         Z = backend.forward([("tok", pending)] + [("tok", d) for d in drafts], n_cached)
         calls += 1
-        P_tgt = np.stack([softmax_T(Z[j], temperature) for j in range(L + 1)])
+        P_tgt = np.stack([softmax_T(Z[j], temperature, top_k) for j in range(L + 1)])
         a, y, _ = verify(P_tgt, Q_dft, drafts, u[L + 1:2 * L + 1], u[2 * L + 1])
         out.extend(drafts[:a] + [y])
         n_cached += 1 + a
@@ -444,7 +467,7 @@ def alg1_two_call(backend, prompt: Sequence[int], L: int, temperature: float,
 
 
 def autoregressive(backend, prompt: Sequence[int], temperature: float, n_tokens: int,
-                   uniform_fn: Callable[[int], float]):
+                   uniform_fn: Callable[[int], float], top_k: int = 0):
     """One token per model call with the KV cache (Baselines)."""
     prompt = [int(t) for t in prompt]
     backend.prefill(prompt[:-1])
@@ -454,7 +477,7 @@ def autoregressive(backend, prompt: Sequence[int], temperature: float, n_tokens:
     for i in range(n_tokens):
         Z = backend.forward([("tok", pending)], n_cached)
         all_logits.append(Z[0])
-        pending = invcdf(softmax_T(Z[0], temperature), uniform_fn(i))
+        pending = invcdf(softmax_T(Z[0], temperature, top_k), uniform_fn(i))
         out.append(pending)
         n_cached += 1
     return out, all_logits

@@ -265,3 +265,90 @@ def test_changing_k_or_temperature_drops_pending_drafts():
     assert len(orc.drafts) == 1
     e, a, info = orc.step(1, 0.5, [0.1] * 3)
     assert info["m"] == 0
+
+
+# ---------------------------------------------------------------- top-k sampling (Experiments, setup)
+def test_top_k_law_against_library_and_special_cases():
+    from scipy.special import softmax
+    rng = np.random.default_rng(3)
+    z = rng.normal(size=50)
+    z[11] = z[40] = z[5]                      # a three-way tie somewhere in the row
+    for T in (1.0, 0.8, 0.2):
+        for k in (1, 2, 10, 49):
+            idx = np.argsort(-z, kind="stable")[:k]          # library sort; stable = lower index first
+            want = np.zeros(50)
+            want[idx] = softmax(z[idx] / T)
+            got = po.softmax_T(z, T, k)
+            np.testing.assert_allclose(got, want, rtol=1e-13, atol=0)
+            assert np.count_nonzero(got) == k and abs(got.sum() - 1.0) < 1e-15
+            assert set(po.top_k_set(z, k).tolist()) == set(idx.tolist())
+    # k >= V and k = 0: no filter; k = 1: the greedy law
+    np.testing.assert_array_equal(po.softmax_T(z, 0.7, 50), po.softmax_T(z, 0.7))
+    np.testing.assert_array_equal(po.softmax_T(z, 0.7, 0), po.softmax_T(z, 0.7))
+    np.testing.assert_array_equal(po.softmax_T(z, 0.7, 1), po.softmax_T(z, 0.0))
+    # a tie across the cut: the lower index stays
+    t = np.array([1.0, 3.0, 3.0, 3.0, 0.0])
+    assert po.top_k_set(t, 2).tolist() == [1, 2]
+    np.testing.assert_allclose(po.softmax_T(t, 1.0, 2), [0, 0.5, 0.5, 0, 0], rtol=1e-15)
+    # greedy is untouched by the filter
+    np.testing.assert_array_equal(po.softmax_T(z, 0.0, 3), po.softmax_T(z, 0.0))
+
+
+# laws whose two largest entries renormalise to dyadic numbers, so that a lattice enumerates them exactly
+TGT_K = [[F(9, 16), F(3, 16), F(1, 8), F(1, 8)],      # top-2 -> [3/4, 1/4, 0, 0]
+         [F(1, 8), F(3, 8), F(3, 8), F(1, 8)],        #       -> [0, 1/2, 1/2, 0]
+         [F(1, 8), F(1, 8), F(3, 16), F(9, 16)],      #       -> [0, 0, 1/4, 3/4]
+         [F(3, 8), F(1, 8), F(1, 8), F(3, 8)]]        #       -> [1/2, 0, 0, 1/2]
+DFT_K = [F(3, 8), F(3, 8), F(1, 8), F(1, 8)]          #       -> [1/2, 1/2, 0, 0]
+
+
+def _filtered(row, k):
+    keep = sorted(range(len(row)), key=lambda i: (-row[i], i))[:k]
+    tot = sum(row[i] for i in keep)
+    return [row[i] / tot if i in keep else F(0) for i in range(len(row))]
+
+
+def test_fused_schedule_with_top_k_emits_the_filtered_target_law_exactly():
+    """Top-2 sampling on vocabulary 4, k = 1 look-ahead: the first two emitted tokens follow
+    P_2(x1) P_2(x2 | x1) with P_2 the top-2 renormalised target law - the filter is applied to
+    target and look-ahead rows alike, and the rejection scheme stays exact for the filtered law."""
+    N = 8
+    prob = np.zeros((2, 4, 4))
+    for t in range(4):
+        prob[0][t] = _np(TGT_K[t])
+        prob[1][t] = _np(DFT_K)
+    assert _filtered(TGT_K[0], 2) == [F(3, 4), F(1, 4), F(0), F(0)]
+    assert _filtered(DFT_K, 2) == [F(1, 2), F(1, 2), F(0), F(0)]
+    first = _filtered(TGT_K[2], 2)
+    want = {}
+    for a in range(4):
+        for b in range(4):
+            v = first[a] * _filtered(TGT_K[a], 2)[b]
+            if v:
+                want[(a, b)] = v
+    law = {}
+    n_two = 0
+    for u1y, u1d, u2a, u2f in itertools.product(lattice(N), repeat=4):
+        orc = po.PassOracle(po.TableBackend(prob), [1, 2])
+        e1, a1, _ = orc.step(1, 1.0, [0.0, u1y, u1d], top_k=2)
+        assert a1 == 0 and len(e1) == 1
+        assert orc.drafts[0] in (0, 1)                       # drafts come from the filtered draft law
+        e2, a2, _ = orc.step(1, 1.0, [u2a, u2f, 0.0])
+        n_two += len(e2) == 2
+        key = (e1[0], e2[0])
+        law[key] = law.get(key, F(0)) + F(1, N ** 4)
+    assert law == want
+    assert n_two > 0
+    # the unfiltered law is a different one
+    assert want != {k: v for k, v in {(a, b): TGT_K[2][a] * TGT_K[a][b] for a in range(4) for b in range(4)}.items() if v}
+
+
+def test_changing_top_k_drops_pending_drafts():
+    prob = _table(2)
+    orc = po.PassOracle(po.TableBackend(prob), [1, 2])
+    orc.step(2, 1.0, [0.1] * 5, top_k=3)
+    assert len(orc.drafts) == 2
+    e, a, info = orc.step(2, 1.0, [0.1] * 5, top_k=2)
+    assert info["m"] == 0 and a == 0 and len(e) == 1
+    e, a, info = orc.step(2, 1.0, [0.1] * 5)                 # top_k stays 2: drafts are used
+    assert info["m"] == 2
