@@ -43,6 +43,8 @@ WORKLOADS = {
     # depth-reduced 7B (same layer shape, 4 layers): small enough for multi-pass ncu captures
     "7b-l4-k4-ctx512-greedy": dict(shape="7b", k=4, prompt=512, T=0.0, batch=1, n_layers=4),
     "7b-k0-ctx512-greedy": dict(shape="7b", k=0, prompt=512, T=0.0, batch=1),
+    # the sampler of the paper's experiments: top-k 10, temperature 0.8
+    "7b-k4-ctx512-T0.8-top10": dict(shape="7b", k=4, prompt=512, T=0.8, batch=1, top_k=10),
 }
 
 
@@ -208,6 +210,7 @@ def main():
     G = max(args.steps + args.warmup, 1) * (k + 1) * 2 + 64
     w = si.make_weights(shape, seed=0, device=dev)
     ctx = pb.PassContext(shape, w, B, P + G + 2 * k + 8, device=dev)
+    ctx.set_top_k(wl.get("top_k", 0))
     for b in range(B):
         ctx.prefill(b, si.make_prompt(shape, P, seq=b + rank * 1000))
     stream = ctx.stream

@@ -170,6 +170,19 @@ int pass_forward_tokens(pass_ctx *ctx, int seq, const int32_t *tokens, int n,
 int pass_reset(pass_ctx *ctx, int seq);
 
 /*
+ * Top-k sampling (Experiments, setup: the sampler behind the paper's timings is top-k with a
+ * temperature).  top_k > 0: in every later step each law - target rows and look-ahead rows alike -
+ * is the temperature softmax over the top_k largest logits of its row, all other tokens have
+ * probability 0; among equal logits the lower token id ranks first.  The filter is applied before
+ * the acceptance ratio and the residual are formed, so the emitted tokens follow the filtered target
+ * law exactly.  top_k = 0 (the default) or top_k >= vocab: no filter.  Greedy steps (temperature 0)
+ * are not affected.  Changing top_k drops pending drafts, like a change of k or temperature.
+ * Host-side setting, no device work.  Errors: INVALID_ARG (ctx NULL, top_k < 0 or > PASS_MAX_TOP_K).
+ */
+#define PASS_MAX_TOP_K 1024
+int pass_set_top_k(pass_ctx *ctx, int top_k);
+
+/*
  * Restore cached keys/values of one layer (e.g. from a saved session): n positions from
  * pos0, k and v as HOST arrays [n][d_model] in cfg.dtype, keys already rotated.  Does not
  * change len; call pass_set_state afterwards.  Errors: INVALID_ARG, CAPACITY, CUDA.

@@ -19,9 +19,11 @@ LIB_PATH = os.path.join(_HERE, "libpass_b200.so")
 PASS_DBG_LOGITS, PASS_DBG_DRAFT_LOGITS, PASS_DBG_KV_LEN, PASS_DBG_N_DRAFT = 0, 1, 2, 3
 PASS_DBG_DRAFTS, PASS_DBG_PENDING, PASS_DBG_N_ACCEPTED, PASS_DBG_STATUS, PASS_DBG_HIDDEN = 4, 5, 6, 7, 8
 PASS_MAX_ROWS = 128
+PASS_MAX_TOP_K = 1024
 
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
+           "pass_set_top_k",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
            "pass_debug_time_linear", "pass_linear_noalloc"]
@@ -71,6 +73,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_step_collect.argtypes = [vp, vp, vp]
     lib.pass_forward_tokens.argtypes = [vp, ci, vp, ci, vp, ci]
     lib.pass_reset.argtypes = [vp, ci]
+    lib.pass_set_top_k.argtypes = [vp, ci]
     lib.pass_set_kv.argtypes = [vp, ci, ci, ci, ci, vp, vp]
     lib.pass_get_kv.argtypes = [vp, ci, ci, ci, ci, vp, vp]
     lib.pass_set_state.argtypes = [vp, ci, ci, ctypes.c_int32]
@@ -187,6 +190,9 @@ class PassContext:
 
     def reset(self, seq: int) -> None:
         _check(self.lib, self.lib.pass_reset(self.h, seq))
+
+    def set_top_k(self, top_k: int) -> None:
+        _check(self.lib, self.lib.pass_set_top_k(self.h, int(top_k)))
 
     def set_state(self, seq: int, length: int, pending: int) -> None:
         _check(self.lib, self.lib.pass_set_state(self.h, seq, length, pending))

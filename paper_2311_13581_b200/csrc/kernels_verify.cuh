@@ -105,11 +105,47 @@ k_verify_stats(VerifyBufs vb, const SeqState* __restrict__ states,
         __syncthreads();
         mx = shf[0];
         for (int w = 1; w < 8; w++) mx = fmaxf(mx, shf[w]);
+        // Top-k sampling (Experiments, setup): the law keeps the top_k largest logits of the row, equal
+        // values ranked by index.  (thr, thr_idx) is the last kept element in that order, found by top_k
+        // rounds of "largest element after the previous one"; every split of the row finds it for itself.
+        float thr = -INFINITY;
+        int thr_idx = V;                                     // keeps everything
+        const int top_k = sp->top_k;
+        if (top_k > 0 && top_k < V) {
+            float lv = INFINITY;
+            int li = -1;
+            for (int it = 0; it < top_k; it++) {
+                float bv = -INFINITY;
+                int bi = V;
+                for (int e = threadIdx.x; e < V; e += kVerifyThreads) {
+                    const float v = z[e];
+                    const bool after = v < lv || (v == lv && e > li);
+                    if (after && (v > bv || (v == bv && e < bi))) { bv = v; bi = e; }
+                }
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                }
+                __syncthreads();                             // shf / shi free
+                if ((threadIdx.x & 31) == 0) { shf[threadIdx.x >> 5] = bv; shi[threadIdx.x >> 5] = bi; }
+                __syncthreads();
+                bv = shf[0];
+                bi = shi[0];
+                for (int w = 1; w < 8; w++)
+                    if (shf[w] > bv || (shf[w] == bv && shi[w] < bi)) { bv = shf[w]; bi = shi[w]; }
+                lv = bv;
+                li = bi;
+            }
+            thr = lv;
+            thr_idx = li;
+        }
         const double invT = 1.0 / (double)T;
         double cs = 0.0;
         for (int e = lo; e < hi; e++) {
             const float v = z[e];
-            const double ev = exp(((double)v - (double)mx) * invT);
+            const bool keep = v > thr || (v == thr && e <= thr_idx);
+            const double ev = keep ? exp(((double)v - (double)mx) * invT) : 0.0;
             vb.E[(size_t)r * V + e] = ev;
             if (la_row) { vb.q_logits[qrow * V + e] = v; vb.q_E[qrow * V + e] = ev; }
             cs += ev;

@@ -154,6 +154,7 @@ struct pass_ctx {
     std::vector<char> prefilled;
     bool have_last = false, params_on_device = false;
     int last_k = -1;
+    int top_k = 0, last_top_k = 0;     // top-k sampling: 0 = off (pass_set_top_k)
     float last_T = -1.f;
     int dev_drop = 0;
     bool pending_collect = false;
@@ -781,6 +782,12 @@ int pass_reset(pass_ctx* c, int seq) {
     return PASS_OK;
 }
 
+int pass_set_top_k(pass_ctx* c, int top_k) {
+    if (!c || top_k < 0 || top_k > PASS_MAX_TOP_K) return PASS_ERR_INVALID_ARG;
+    c->top_k = top_k;
+    return PASS_OK;
+}
+
 int pass_set_state(pass_ctx* c, int seq, int len, int32_t pending) {
     if (!c || seq < 0 || seq >= c->md.B || len < 0 || pending < 0 || pending >= c->md.V) return PASS_ERR_INVALID_ARG;
     if (len > c->md.cap) return PASS_ERR_CAPACITY;
@@ -857,19 +864,20 @@ static int step_checks(pass_ctx* c, int k, float T, const void* uniforms) {
 
 static int step_launch(pass_ctx* c, int k, float T) {
     // step parameters: only re-sent when they differ from what the device holds
-    const int drop = (c->have_last && (k != c->last_k || T != c->last_T)) ? 1 : 0;
-    if (!c->params_on_device || !c->have_last || k != c->last_k || T != c->last_T || drop != c->dev_drop) {
+    const bool changed = k != c->last_k || T != c->last_T || c->top_k != c->last_top_k;
+    const int drop = (c->have_last && changed) ? 1 : 0;
+    if (!c->params_on_device || !c->have_last || changed || drop != c->dev_drop) {
         if (c->ring_pos == kParamRing) {
             CUDA_TRY(cudaStreamSynchronize(c->stream));
             c->ring_pos = 0;
         }
         StepParams* p = c->pin_params + c->ring_pos++;
-        p->temperature = T; p->k = k; p->drop_drafts = drop; p->pad_ = 0;
+        p->temperature = T; p->k = k; p->drop_drafts = drop; p->top_k = c->top_k;
         CUDA_TRY(cudaMemcpyAsync(c->d_params, p, sizeof(StepParams), cudaMemcpyHostToDevice, c->stream));
         c->params_on_device = true;
         c->dev_drop = drop;
     }
-    c->have_last = true; c->last_k = k; c->last_T = T;
+    c->have_last = true; c->last_k = k; c->last_T = T; c->last_top_k = c->top_k;
     c->launches = 0;
     if (c->use_graph) {
         auto it = c->graphs.find(k);

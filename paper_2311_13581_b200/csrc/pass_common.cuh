@@ -40,8 +40,8 @@ struct SeqState {
 struct StepParams {
     float temperature;
     int k;
-    int drop_drafts;   // k or temperature changed: pending drafts are void
-    int pad_;
+    int drop_drafts;   // k, temperature or top_k changed: pending drafts are void
+    int top_k;         // > 0: every law is the softmax over the top_k largest logits of its row only
     // followed by float u[max_batch][kUSlots]
 };
 

@@ -25,8 +25,11 @@ def logits_error(Zg, Zo, fp32):
     return float(np.max(num / den))
 
 
-def lockstep(ctx, oracles, k, T, n_steps, seed=0, step0=0, cdf_tol_A=1e-4, check_A=True):
+def lockstep(ctx, oracles, k, T, n_steps, seed=0, step0=0, cdf_tol_A=1e-4, check_A=True, top_k=0):
     B, V, M = ctx.B, ctx.vocab, 1 + 2 * k
+    ctx.set_top_k(top_k)
+    for orc in oracles:
+        orc.top_k = top_k
     T = float(np.float32(T))            # the library takes the temperature as a C float
     fp32 = ctx.shape.dtype == "fp32"
     stats = {"steps": 0, "tokens": 0, "accepted": 0, "max_logit_err": 0.0, "A_excused": 0,
@@ -53,7 +56,7 @@ def lockstep(ctx, oracles, k, T, n_steps, seed=0, step0=0, cdf_tol_A=1e-4, check
             assert 1 <= len(g_em) <= k + 1 and len(g_em) == n_out[b] == n_acc[b] + 1
             # level B: float64 verify on the library's own logits
             if m:
-                Qg = np.stack([po.softmax_T(prev_la[b][t], T) for t in range(m)])
+                Qg = np.stack([po.softmax_T(prev_la[b][t], T, top_k) for t in range(m)])
             else:
                 Qg = np.zeros((0, V))
             decB = orc.decide(Zg, Qg, k, T, u[b])
@@ -82,7 +85,7 @@ def lockstep(ctx, oracles, k, T, n_steps, seed=0, step0=0, cdf_tol_A=1e-4, check
                 else:
                     stats["A_mismatch"] += 1
             # adopt the library's outcome
-            Qn = np.stack([po.softmax_T(Zo[m + 1 + t], T) for t in range(k)]) if g_nd else np.zeros((0, V))
+            Qn = np.stack([po.softmax_T(Zo[m + 1 + t], T, top_k) for t in range(k)]) if g_nd else np.zeros((0, V))
             orc.commit(g_em, g_nd, Qn)
             if g_nd:
                 prev_la[b] = Zg[m + 1:m + 1 + k].copy()

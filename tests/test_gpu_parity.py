@@ -140,6 +140,64 @@ def test_changing_k_and_temperature_between_steps(tiny_w):
     ctx.close()
 
 
+# ------------------------------------------------------------------ top-k sampling
+@pytest.mark.parametrize("top_k,T", [(10, 0.8), (25, 0.5), (1, 1.0), (3, 0.2)])
+def test_tiny_fp32_top_k_sampling(tiny_w, top_k, T):
+    """Top-k sampling (the sampler of the paper's experiments, k = 10 / 25): the filter decides which
+    tokens can be emitted at all, so every emitted token and every draft must lie in the top-k set of
+    its row, and the decisions must agree with the float64 rule on the same logits."""
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY, 20)
+    ctx, oracles, _ = make_pair(TINY, 1, 160, [prompt], weights=tiny_w)
+    stats, streams = lockstep(ctx, oracles, 2, T, 12, top_k=top_k)
+    assert stats["max_logit_err"] <= 1e-3, stats
+    assert stats["tokens"] >= 12
+    if top_k == 1:
+        # top-1 sampling is greedy decoding whatever the temperature and the uniforms
+        ctx2, oracles2, _ = make_pair(TINY, 1, 160, [prompt], weights=tiny_w)
+        _, greedy = lockstep(ctx2, oracles2, 2, 0.0, 12)
+        n = min(len(greedy[0]), len(streams[0]))
+        assert streams[0][:n] == greedy[0][:n]
+        ctx2.close()
+    ctx.close()
+
+
+def test_top_k_changes_between_steps_and_batch(tiny_w):
+    from parity_util import lockstep, make_pair
+    prompts = [si.make_prompt(TINY, 14, seed=s) for s in (0, 1, 2)]
+    ctx, oracles, _ = make_pair(TINY, 3, 160, prompts, weights=tiny_w)
+    step = 0
+    for top_k in (0, 10, 10, 4, 0):
+        stats, _ = lockstep(ctx, oracles, 2, 0.9, 3, step0=step, top_k=top_k)
+        step += 3
+        assert stats["max_logit_err"] <= 1e-3
+    with pytest.raises(_pb().PassError):
+        ctx.set_top_k(-1)
+    with pytest.raises(_pb().PassError):
+        ctx.set_top_k(_pb().PASS_MAX_TOP_K + 1)
+    ctx.close()
+
+
+def test_7b_layer_shape_top_k_10():
+    """The paper's sampler (top-k 10, temperature 0.8) at the 7B layer shape, vocabulary 32000."""
+    import paper_2311_13581_b200 as pb
+    from parity_util import lockstep
+    shape = SEVENB_2L
+    w = si.make_weights(shape, seed=0, device="cuda:0")
+    w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
+    ctx_len, cap = 600, 700
+    ctx = pb.PassContext(shape, w, 1, cap)
+    be = po.TransformerBackend(shape, w_cpu, cap)
+    _load_synthetic_cache(ctx, [be], shape, ctx_len)
+    ctx.set_state(0, ctx_len, 11)
+    orc = po.PassOracle.__new__(po.PassOracle)
+    orc.be, orc.len, orc.pending, orc.drafts = be, ctx_len, 11, []
+    orc.Q_dft, orc.k_prev, orc.T_prev, orc.last_logits = np.zeros((0, shape.vocab)), None, None, None
+    stats, _ = lockstep(ctx, [orc], 4, 0.8, 4, check_A=False, top_k=10)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
 # ------------------------------------------------------------------ errors never fault
 def test_error_paths(tiny_w):
     pb = _pb()
