@@ -207,7 +207,8 @@ def main():
     dev = f"cuda:{local}"
     torch.cuda.set_device(local)
     k, T, B, P = wl["k"], wl["T"], wl["batch"], wl["prompt"]
-    G = max(args.steps + args.warmup, 1) * (k + 1) * 2 + 64
+    n_two = 16 if k > 0 else 0                                   # iterations of the two-call schedule, reported beside
+    G = max(args.steps + args.warmup, 1) * (k + 1) * 2 + 64 + n_two * (k + 2)
     w = si.make_weights(shape, seed=0, device=dev)
     ctx = pb.PassContext(shape, w, B, P + G + 2 * k + 8, device=dev)
     ctx.set_top_k(wl.get("top_k", 0))
@@ -262,6 +263,22 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- Algorithm 1 as printed (two model calls per iteration), for the tokens-per-call comparison
+    two_call = None
+    if n_two:
+        u2 = np.stack([np.stack([si.step_uniforms(rank + 77, b, it, 2 * k + 2).numpy() for b in range(B)])
+                       for it in range(n_two)])
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        tok2 = 0
+        for it in range(n_two):
+            _, n2 = ctx.step_two_call(k, T, u2[it] if T > 0 else None)
+            tok2 += int(n2.sum())
+        torch.cuda.synchronize()
+        dt2 = time.perf_counter() - t0
+        two_call = {"iterations": n_two, "model_calls": 2 * n_two, "tokens_per_call": tok2 / (2 * n_two * B),
+                    "ms_per_call": dt2 * 1e3 / (2 * n_two), "timing": "host clock, through pass_step_two_call"}
+
     # ---- the dominant kernel by itself: the GEMM chain of one layer (O-proj -> gate|up -> down -> next QKV),
     # 64 launches back to back cycling over the layers (every launch streams other weights), CUDA events on
     # the library's stream.  Last, because it scribbles over the residual stream and one cache row.
@@ -289,6 +306,8 @@ def main():
                    "l2": "per-step weight stream (%.1f GB) exceeds L2" % (weight_bytes(shape) / 1e9),
                    "replicas": world},
         "tokens_per_step": tokens / (args.steps * world),
+        "schedules": {"fused_one_call": {"tokens_per_call": tokens / (args.steps * world * B)},
+                      "algorithm1_two_call": two_call},
         "hbm_gbs": gbs, "frac_of_8tbs": gbs / 8000.0,
         "gpu_launches": launches,
         "clocks": clocks,

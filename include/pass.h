@@ -142,6 +142,24 @@ int pass_step(pass_ctx *ctx, int k_lookahead, float temperature, const float *un
               int32_t *out_tokens, int32_t *n_out);
 
 /*
+ * One iteration of Algorithm 1 AS PRINTED (Parallel Speculative Sampling: two model calls per
+ * iteration) for all sequences, on the same kernels as pass_step:
+ *   drafting call   rows [pending, LA_1..LA_L]: x_{n+1} ~ softmax(logits_0 / T) and the drafts
+ *                   d_t ~ Q_t = softmax(logits_t / T); pending drafts of an earlier fused step are dropped;
+ *   validation call rows [x_{n+1}, d_1..d_L]: accept tests, residual or extra token as in pass_step;
+ *                   the call still carries L look-ahead rows (a step has 1+2L rows whatever it does,
+ *                   and its time is set by the weights, not by the rows) whose outputs are not used.
+ *   uniforms   : [max_batch][2L+2] floats in [0,1): slot 0 samples x_{n+1}, slots 1..L the drafts,
+ *                slots L+1..2L the accept tests, slot 2L+1 the final token.  NULL iff temperature == 0.
+ *   out_tokens : [max_batch][k_max+2] int32: x_{n+1}, the accepted drafts, the final token.
+ *   n_out      : [max_batch] int32: 2 .. L+2 (each call adds at least one token).
+ * Exists so that both schedules can be stated side by side (tokens per model call); pass_step's
+ * one-call form is the fast path.  Synchronises the stream twice.  Errors: as pass_step.
+ */
+int pass_step_two_call(pass_ctx *ctx, int L, float temperature, const float *uniforms,
+                       int32_t *out_tokens, int32_t *n_out);
+
+/*
  * The same iteration without host round trip: reads the uniforms from DEVICE memory
  * (same layout, may be NULL iff temperature == 0), enqueues the step and returns at once.
  * Results stay on the device until pass_step_collect.  Capacity is checked against an

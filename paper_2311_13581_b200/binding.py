@@ -23,7 +23,7 @@ PASS_MAX_TOP_K = 1024
 
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
-           "pass_set_top_k",
+           "pass_set_top_k", "pass_step_two_call",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
            "pass_debug_time_linear", "pass_linear_noalloc"]
@@ -69,6 +69,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_load_weights.argtypes = [vp, ctypes.POINTER(_Weights)]
     lib.pass_prefill.argtypes = [vp, ci, vp, ci]
     lib.pass_step.argtypes = [vp, ci, cf, vp, vp, vp]
+    lib.pass_step_two_call.argtypes = [vp, ci, cf, vp, vp, vp]
     lib.pass_step_enqueue.argtypes = [vp, ci, cf, vp]
     lib.pass_step_collect.argtypes = [vp, vp, vp]
     lib.pass_forward_tokens.argtypes = [vp, ci, vp, ci, vp, ci]
@@ -190,6 +191,20 @@ class PassContext:
 
     def reset(self, seq: int) -> None:
         _check(self.lib, self.lib.pass_reset(self.h, seq))
+
+    def step_two_call(self, L: int, temperature: float, uniforms):
+        """uniforms: numpy float32 [B][2L+2] or None (greedy). Returns (list of emitted lists, n_out)."""
+        out = np.zeros((self.B, self.k_max + 2), dtype=np.int32)
+        n_out = np.zeros(self.B, dtype=np.int32)
+        if uniforms is not None:
+            uniforms = np.ascontiguousarray(uniforms, dtype=np.float32)
+            assert uniforms.shape == (self.B, 2 * L + 2)
+            up = uniforms.ctypes.data
+        else:
+            up = None
+        _check(self.lib, self.lib.pass_step_two_call(self.h, int(L), ctypes.c_float(temperature), up,
+                                                     out.ctypes.data, n_out.ctypes.data))
+        return [out[b, :n_out[b]].tolist() for b in range(self.B)], n_out
 
     def set_top_k(self, top_k: int) -> None:
         _check(self.lib, self.lib.pass_set_top_k(self.h, int(top_k)))

@@ -280,7 +280,7 @@ k_verify_decide(VerifyBufs vb, SeqState* __restrict__ states, const StepParams* 
             st.n_acc = a;
             st.kv_len += a + 1;
             st.pending = y;
-            if (a == m && k > 0) {
+            if (a == m && k > 0 && !sp->validate_only) {
                 for (int t = 0; t < k; t++) st.drafts[t] = s_arg[m + 1 + t];
                 st.m = k;
                 st.q_sel ^= 1;
@@ -350,7 +350,7 @@ k_verify_decide(VerifyBufs vb, SeqState* __restrict__ states, const StepParams* 
         y = block_invcdf(vb.chunk + (size_t)(r0 + m) * kChunks, V, (double)u[k], wp, sh_d, sh_i);
     }
     int nd[kMaxLA];
-    if (a == m) {
+    if (a == m && !sp->validate_only) {
         for (int t = 0; t < k; t++) {
             const double* Eq = vb.E + (size_t)(r0 + m + 1 + t) * V;
             auto wq = [&](int e) { return Eq[e]; };
@@ -365,7 +365,7 @@ k_verify_decide(VerifyBufs vb, SeqState* __restrict__ states, const StepParams* 
         st.n_acc = a;
         st.kv_len += a + 1;
         st.pending = y;
-        if (a == m && k > 0) {
+        if (a == m && k > 0 && !sp->validate_only) {
             for (int t = 0; t < k; t++) st.drafts[t] = nd[t];
             st.m = k;
             st.q_sel ^= 1;

@@ -155,6 +155,8 @@ struct pass_ctx {
     bool have_last = false, params_on_device = false;
     int last_k = -1;
     int top_k = 0, last_top_k = 0;     // top-k sampling: 0 = off (pass_set_top_k)
+    int validate_only = 0, dev_validate_only = 0;   // two-call schedule: the current call is a validation call
+    bool force_drop = false;           // two-call schedule: the drafting call starts without pending drafts
     float last_T = -1.f;
     int dev_drop = 0;
     bool pending_collect = false;
@@ -865,17 +867,20 @@ static int step_checks(pass_ctx* c, int k, float T, const void* uniforms) {
 static int step_launch(pass_ctx* c, int k, float T) {
     // step parameters: only re-sent when they differ from what the device holds
     const bool changed = k != c->last_k || T != c->last_T || c->top_k != c->last_top_k;
-    const int drop = (c->have_last && changed) ? 1 : 0;
-    if (!c->params_on_device || !c->have_last || changed || drop != c->dev_drop) {
+    const int drop = ((c->have_last && changed) || c->force_drop) ? 1 : 0;
+    if (!c->params_on_device || !c->have_last || changed || drop != c->dev_drop ||
+        c->validate_only != c->dev_validate_only) {
         if (c->ring_pos == kParamRing) {
             CUDA_TRY(cudaStreamSynchronize(c->stream));
             c->ring_pos = 0;
         }
         StepParams* p = c->pin_params + c->ring_pos++;
         p->temperature = T; p->k = k; p->drop_drafts = drop; p->top_k = c->top_k;
+        p->validate_only = c->validate_only; p->pad_[0] = p->pad_[1] = p->pad_[2] = 0;
         CUDA_TRY(cudaMemcpyAsync(c->d_params, p, sizeof(StepParams), cudaMemcpyHostToDevice, c->stream));
         c->params_on_device = true;
         c->dev_drop = drop;
+        c->dev_validate_only = c->validate_only;
     }
     c->have_last = true; c->last_k = k; c->last_T = T; c->last_top_k = c->top_k;
     c->launches = 0;
@@ -965,6 +970,45 @@ int pass_step(pass_ctx* c, int k, float T, const float* uniforms, int32_t* out_t
     rc = step_launch(c, k, T);
     if (rc != PASS_OK) return rc;
     return pass_step_collect(c, out_tokens, n_out);
+}
+
+int pass_step_two_call(pass_ctx* c, int L, float T, const float* uniforms, int32_t* out_tokens, int32_t* n_out) {
+    if (!c || !out_tokens || !n_out || L < 0 || L > c->md.k_max) return PASS_ERR_INVALID_ARG;
+    if (!uniforms && T != 0.f) return PASS_ERR_INVALID_ARG;
+    const int B = c->md.B, km = c->md.k_max, nu = 2 * L + 2;
+    std::vector<float> u1((size_t)B * (2 * L + 1), 0.f), u2((size_t)B * (2 * L + 1), 0.f);
+    std::vector<int32_t> t1((size_t)B * (km + 1)), t2((size_t)B * (km + 1)), n1(B), n2(B);
+    if (uniforms) {
+        for (int b = 0; b < B; b++) {
+            const float* U = uniforms + (size_t)b * nu;
+            for (int j = 0; j < nu; j++)
+                if (!(U[j] >= 0.f && U[j] < 1.f)) return PASS_ERR_INVALID_ARG;
+            float* a = u1.data() + (size_t)b * (2 * L + 1);
+            float* v = u2.data() + (size_t)b * (2 * L + 1);
+            a[L] = U[0];                                         // x_{n+1}
+            for (int t = 0; t < L; t++) a[L + 1 + t] = U[1 + t];  // drafts
+            for (int j = 0; j < L; j++) v[j] = U[L + 1 + j];      // accept tests
+            v[L] = U[2 * L + 1];                                  // residual / extra token
+        }
+    }
+    // drafting call: [x_n, LA_1..LA_L], no pending drafts
+    c->force_drop = true;
+    c->validate_only = 0;
+    int rc = pass_step(c, L, T, uniforms ? u1.data() : nullptr, t1.data(), n1.data());
+    c->force_drop = false;
+    if (rc != PASS_OK) return rc;
+    // validation call: [x_{n+1}, d_1..d_L]
+    c->validate_only = 1;
+    rc = pass_step(c, L, T, uniforms ? u2.data() : nullptr, t2.data(), n2.data());
+    c->validate_only = 0;
+    if (rc != PASS_OK) return rc;
+    for (int b = 0; b < B; b++) {
+        int32_t* o = out_tokens + (size_t)b * (km + 2);
+        o[0] = t1[(size_t)b * (km + 1)];
+        for (int j = 0; j < n2[b]; j++) o[1 + j] = t2[(size_t)b * (km + 1) + j];
+        n_out[b] = 1 + n2[b];
+    }
+    return PASS_OK;
 }
 
 static int kv_copy(pass_ctx* c, int seq, int layer, int pos0, int n, void* k, void* v, int gather) {

@@ -42,6 +42,8 @@ struct StepParams {
     int k;
     int drop_drafts;   // k, temperature or top_k changed: pending drafts are void
     int top_k;         // > 0: every law is the softmax over the top_k largest logits of its row only
+    int validate_only; // 1: validation call of the two-call schedule - the look-ahead rows' outputs are not used
+    int pad_[3];
     // followed by float u[max_batch][kUSlots]
 };
 

@@ -198,6 +198,50 @@ def test_7b_layer_shape_top_k_10():
     ctx.close()
 
 
+# ------------------------------------------------------------------ Algorithm 1 as printed (two calls)
+@pytest.mark.parametrize("L,T,top_k", [(2, 1.0, 0), (4, 0.0, 0), (1, 0.7, 0), (3, 0.9, 5)])
+def test_two_call_schedule_matches_algorithm_1_of_the_oracle(tiny_w, L, T, top_k):
+    """pass_step_two_call against the oracle's transcription of Algorithm 1: same prompt, same
+    uniforms per iteration, token streams compared one by one.  The two sides compute their logits
+    apart (float32 kernels / float64), so a decision that sits within 1e-4 of a boundary on the
+    oracle's side may differ; the comparison stops there (it did not happen with these seeds)."""
+    from parity_util import make_pair
+    prompt = si.make_prompt(TINY, 18)
+    n_it = 14
+    ctx, _, _ = make_pair(TINY, 1, 200, [prompt], weights=tiny_w)
+    ctx.set_top_k(top_k)
+    Tf = float(np.float32(T))
+    U = [si.step_uniforms(5, 0, it, 2 * L + 2).numpy() for it in range(n_it)]
+    gpu, calls = [], 0
+    for it in range(n_it):
+        em, n_out = ctx.step_two_call(L, Tf, None if T == 0 else U[it][None])
+        assert 2 <= len(em[0]) == n_out[0] <= L + 2
+        gpu += em[0]
+        calls += 2
+    be = po.TransformerBackend(TINY, tiny_w, 200)
+    want, ocalls = po.alg1_two_call(be, prompt, L, Tf, len(gpu), lambda it, n: U[it] if it < n_it else np.zeros(n),
+                                    top_k=top_k)
+    n = min(len(want), len(gpu))
+    assert gpu[:n] == want[:n]
+    assert n >= 2 * n_it
+    # the gain of the two-call scheme is bounded by (L + 2) / 2 tokens per call
+    assert len(gpu) / calls <= (L + 2) / 2
+    ctx.close()
+
+
+def test_unk_lookahead_baseline_runs_through_the_same_path():
+    """The paper's ablation feeds one fixed token embedding as every look-ahead input: that is a
+    look-ahead table whose rows are all equal - same kernels, same parity."""
+    from parity_util import lockstep, make_pair
+    w = si.make_weights(TINY, seed=0)
+    w["la_emb"][:] = w["tok_emb"][0]
+    prompt = si.make_prompt(TINY, 16)
+    ctx, oracles, _ = make_pair(TINY, 1, 160, [prompt], weights=w)
+    stats, _ = lockstep(ctx, oracles, 3, 1.0, 8)
+    assert stats["max_logit_err"] <= 1e-3, stats
+    ctx.close()
+
+
 # ------------------------------------------------------------------ errors never fault
 def test_error_paths(tiny_w):
     pb = _pb()
