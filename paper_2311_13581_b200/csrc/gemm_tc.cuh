@@ -53,7 +53,8 @@ struct GemmParams {
     const void* w_base[3];         // the weight matrices behind maps 0..2 (for L2 prefetch), [w_rows][w_ld] bf16
     int w_rows[3];
     int w_ld;
-    float* partial_ws;             // [gridDim][2][rh][128] fp32
+    float* partial_ws;             // [gridDim][2][rh][128] fp32: more than 16 rows (arrival counter per tile)
+    float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: up to 16 rows
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
     // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
@@ -395,6 +396,69 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             }
         }
     }
+}
+
+// Partial sums of up to 16 token rows are handed over without a counter: a slot word is either EMPTY (all
+// bits set - a NaN pattern that fp32 arithmetic never produces, it makes the canonical 0x7fffffff) or a
+// value.  Contributors just store their values; the finisher loads the words it needs and repeats the
+// load until none of them is empty; when it is done with a tile it stores EMPTY back, so every launch
+// finds the slots as the first one did (the workspace is filled with 0xff bytes when it is created).
+// A 4-byte word is written and read in one piece, hence no fence, no arrival counter and no second trip
+// to L2.  Slot layout [row][feature].  Should a value ever come out as the EMPTY pattern, the finisher
+// runs into its bounded wait and the launch reports a time-out; nothing is consumed silently.
+constexpr uint32_t kEmptyWord = 0xFFFFFFFFu;
+__device__ __forceinline__ void st_word(float* p, uint32_t w) {
+    asm volatile("st.relaxed.gpu.global.b32 [%0], %1;" ::"l"(p), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_word(const float* p) {
+    uint32_t w;
+    asm volatile("ld.relaxed.gpu.global.b32 %0, [%1];" : "=r"(w) : "l"(p) : "memory");
+    return w;
+}
+constexpr int kLLRows = 9;          // rows fetched per trip (1 + 2k rows of k = 4 look-ahead tokens)
+constexpr int kLLPeers = 5;         // other contributors fetched per trip
+
+// acc[j] += value of row row0 + j from each of `n_others` contributors (slots `first` + q * stride, k order),
+// for this thread's feature.  Spins (bounded) until no word is EMPTY, then marks the words EMPTY again if
+// `reset`.  Returns false on time-out.
+__device__ __forceinline__ bool ll_gather(float* first, size_t stride, int n_others, int row0, int nrows,
+                                          float (&acc)[kLLRows], volatile int* s_abort, int* g_status) {
+    bool fine = true;
+    for (int q0 = 0; q0 < n_others; q0 += kLLPeers) {
+        uint32_t w[kLLPeers][kLLRows];
+        const long long t0 = clock64();
+        for (;;) {
+            bool ok = true;
+#pragma unroll
+            for (int qq = 0; qq < kLLPeers; qq++) {
+                const float* src = first + (size_t)(q0 + qq) * stride + (size_t)row0 * kTileN;
+#pragma unroll
+                for (int j = 0; j < kLLRows; j++)
+                    w[qq][j] = (q0 + qq < n_others && j < nrows) ? ld_word(src + (size_t)j * kTileN) : 0u;
+            }
+#pragma unroll
+            for (int qq = 0; qq < kLLPeers; qq++)
+#pragma unroll
+                for (int j = 0; j < kLLRows; j++) ok &= w[qq][j] != kEmptyWord;
+            if (ok) break;
+            if (*s_abort || clock64() - t0 > kWaitCycles) {
+                *s_abort = 1;
+                atomicOr(g_status, kStatusTimeout);
+                fine = false;
+                break;
+            }
+        }
+#pragma unroll
+        for (int qq = 0; qq < kLLPeers; qq++)
+#pragma unroll
+            for (int j = 0; j < kLLRows; j++) acc[j] += __uint_as_float(w[qq][j]);
+    }
+    return fine;
+}
+// the words ll_gather consumed become EMPTY again (after the tile's results are out: off the critical path)
+__device__ __forceinline__ void ll_reset(float* first, size_t stride, int n_others, int nrows) {
+    for (int q = 0; q < n_others; q++)
+        for (int j = 0; j < nrows; j++) st_word(first + (size_t)q * stride + (size_t)j * kTileN, kEmptyWord);
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -742,7 +806,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
                 float2 cs_pre[16] = {};
-                const bool pre = p.rh == 16 && pc.n_pieces > 1;
+                const bool pre = p.rh == 16 && pc.n_pieces > 1 && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
@@ -759,8 +823,83 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 if (*(volatile int*)&s_epi_fail) { ok = false; break; }
                 if (et == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
-                const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
                 const bool whole = pc.n_pieces == 1;
+                const bool ll = p.rh == 16 && !whole;          // counter-free hand-over of the partial sums, fixed finisher
+                float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
+                int ll_n = 0;
+                const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
+                bool tile_done = whole;
+                if (ll) {
+                    float av[16];
+#pragma unroll
+                    for (int c0 = 0; c0 < 16; c0 += 8) {
+                        float hi[8], lo[8];
+                        tmem_ld8(t_addr + c0, hi);
+                        tmem_ld8(t_addr + 16 + c0, lo);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 8; j++) av[c0 + j] = hi[j] + lo[j];
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+                    if (pc.index != 0) {
+                        // a later part of the tile: hand it to the CTA that holds the tile's first k-blocks
+                        float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
+#pragma unroll
+                        for (int j = 0; j < 16; j++)
+                            if (j < p.R) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
+                    } else {
+                        // The tile's first part is this CTA's LAST piece of the GEMM (its range ends inside the
+                        // tile), so it is the natural finisher: the other parts were either computed at the very
+                        // start of their CTAs' ranges or finish together with this one.
+                        tile_done = true;
+                        const int n = pc.tile * kTileN + ec.lane_in_tile;
+                        float hv[2][8] = {};
+                        if (p.epi == kEpiResid) {
+#pragma unroll
+                            for (int j = 0; j < 16; j++)
+                                hv[j >> 3][j & 7] = (j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
+                        }
+                        // every contributor but the first keeps its part in slot 0 (its range begins inside the tile)
+                        float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
+                        const size_t peer_stride = 2 * slot_floats;
+                        float acc9[kLLRows];
+#pragma unroll
+                        for (int j = 0; j < kLLRows; j++) acc9[j] = av[j];
+                        ll_gather(peer, peer_stride, pc.n_pieces - 1, 0, min(p.R, kLLRows), acc9, &s_abort, cp.status);
+                        if (et == 0) PASS_TRACE(oi, 5);
+                        // both halves run through ONE copy of the epilogue code (the loop is kept rolled)
+#pragma unroll 1
+                        for (int half = 0; half < 2; half++) {
+                            if (half * 8 >= p.R) break;
+                            float a8[8], h8[8];
+                            float2 cs8[8];
+                            if (half == 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; j++) a8[j] = acc9[j];
+                            } else {
+                                float rest[kLLRows];
+#pragma unroll
+                                for (int j = 0; j < kLLRows; j++) rest[j] = j < 7 ? av[9 + j] : 0.f;
+                                if (p.R > kLLRows)
+                                    ll_gather(peer, peer_stride, pc.n_pieces - 1, kLLRows, p.R - kLLRows, rest, &s_abort, cp.status);
+                                a8[0] = acc9[8];
+#pragma unroll
+                                for (int j = 1; j < 8; j++) a8[j] = rest[j - 1];
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; j++) {
+                                h8[j] = half ? hv[1][j] : hv[0][j];
+                                cs8[j] = half ? cs_pre[8 + j] : cs_pre[j];
+                            }
+                            epi_store(p, ec, pc.tile, half * 8, a8, p.epi == kEpiResid ? h8 : nullptr,
+                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs8 : nullptr);
+                        }
+                        ll_peer = peer;
+                        ll_n = pc.n_pieces - 1;
+                    }
+                } else {
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
                 for (int c0 = 0; c0 < p.rh; c0 += 8) {
                     float hi[8], lo[8];
@@ -782,11 +921,11 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
-                bool tile_done = whole;
                 if (!whole) {
-                    // The last CTA to deliver its part of the tile sums all parts in k order.  The barrier
-                    // orders every thread's partial stores before thread 0's acq_rel atomic (release is
-                    // cumulative), and the loads after the second barrier behind its acquire.
+                    // More than 16 rows (prompt chunks): the last CTA to deliver its part of the tile sums all
+                    // parts in k order.  The barrier orders every thread's partial stores before thread 0's
+                    // acq_rel atomic (release is cumulative), and the loads after the second barrier behind
+                    // its acquire.
                     epi_bar();
                     if (et == 0) {
                         int prev;
@@ -801,63 +940,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         tile_done = true;
                         const int c_first = cta - pc.index;
                         const int slot_first = pc.first_slot;
-                        if (p.rh == 16) {
-                            // the common case (up to 16 rows): both 8-row halves in one pass.  The residual
-                            // values and the parts of four contributors are requested together, so the whole
-                            // reduction costs one or two trips to L2 instead of one per half and contributor group.
-                            const int n = pc.tile * kTileN + ec.lane_in_tile;
-                            float hv[2][8] = {};
-                            if (p.epi == kEpiResid) {
-#pragma unroll
-                                for (int j = 0; j < 16; j++)
-                                    hv[j >> 3][j & 7] = (j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
-                            }
-                            float acc[2][8];
-#pragma unroll
-                            for (int j = 0; j < 16; j++) acc[j >> 3][j & 7] = 0.f;
-                            // up to six contributors per trip (the 7B/13B shapes never have more on a tile)
-                            // and only the float4s that hold real rows
-                            const int nf4 = (p.R + 3) >> 2;
-                            for (int q0 = 0; q0 < pc.n_pieces; q0 += 6) {
-                                float4 v[6][4];
-#pragma unroll
-                                for (int qq = 0; qq < 6; qq++) {
-                                    const int qi = min(q0 + qq, pc.n_pieces - 1);
-                                    const int cq = c_first + qi;
-                                    const int slot = qi == 0 ? slot_first : 0;
-                                    const float4* src = reinterpret_cast<const float4*>(
-                                        p.partial_ws + ((size_t)cq * 2 + slot) * slot_floats) + ec.lane_in_tile;
-#pragma unroll
-                                    for (int f = 0; f < 4; f++)
-                                        v[qq][f] = (f < nf4 && q0 + qq < pc.n_pieces) ? __ldcg(src + f * kTileN) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                }
-#pragma unroll
-                                for (int qq = 0; qq < 6; qq++) {
-#pragma unroll
-                                    for (int f = 0; f < 4; f++) {
-                                        acc[f >> 1][(f & 1) * 4 + 0] += v[qq][f].x; acc[f >> 1][(f & 1) * 4 + 1] += v[qq][f].y;
-                                        acc[f >> 1][(f & 1) * 4 + 2] += v[qq][f].z; acc[f >> 1][(f & 1) * 4 + 3] += v[qq][f].w;
-                                    }
-                                }
-                            }
-                            // both halves run through ONE copy of the epilogue code (the loop is kept rolled):
-                            // this code runs once per GEMM and CTA, so every instruction line of it is a
-                            // fetch from L2, and a second inlined copy would pay for its lines again
-#pragma unroll 1
-                            for (int half = 0; half < 2; half++) {
-                                if (half * 8 >= p.R) break;
-                                float a8[8], h8[8];
-                                float2 cs8[8];
-#pragma unroll
-                                for (int j = 0; j < 8; j++) {
-                                    a8[j] = half ? acc[1][j] : acc[0][j];
-                                    h8[j] = half ? hv[1][j] : hv[0][j];
-                                    cs8[j] = half ? cs_pre[8 + j] : cs_pre[j];
-                                }
-                                epi_store(p, ec, pc.tile, half * 8, a8, p.epi == kEpiResid ? h8 : nullptr,
-                                          p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs8 : nullptr);
-                            }
-                        } else
                         for (int c0 = 0; c0 < p.rh; c0 += 8) {
                             float acc[8];
 #pragma unroll
@@ -889,6 +971,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         }
                     }
                 }
+                }
                 if (et == 0 && tile_done && !whole) PASS_TRACE(oi, 6);
                 if (signal && tile_done) {
                     // every thread's stores of this tile happen-before thread 0's release (barrier + cumulativity)
@@ -897,6 +980,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cp.op_done + oi) : "memory");
                     if (et == 0) PASS_TRACE(oi, 7);
                 }
+                if (ll_peer) ll_reset(ll_peer, 2 * slot_floats, ll_n, p.R);
             }
             if (et == 0) *(volatile int*)&s_epi_done = oi;
             if (et == 0) PASS_TRACE(oi, 3);

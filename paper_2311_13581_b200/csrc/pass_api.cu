@@ -18,6 +18,7 @@ using namespace pass;
 namespace {
 
 constexpr int kMaxCtas = 160;      // upper bound of CTAs of one GEMM launch (one per SM)
+constexpr size_t kLLRegionBytes = (size_t)(kMaxCtas + 1) * 2 * 16 * 128 * 4;   // per GEMM of a chain; +1: CTA c reads c+1..
 
 struct Carve {
     size_t off = 0;
@@ -33,6 +34,7 @@ struct Layout {
     size_t h, xn, qkv, attn, gu, act, logits;
     size_t E, chunk, row_sum, row_max, amax_val, amax_idx, q_logits, q_E, q_sum, scratch;
     size_t xn_bf, attn_bf, act_bf, q_out, sumsq_a, sumsq_b, partial_ws, counters;   // tensor-core path
+    size_t ll_ws;
     size_t attn_po, attn_pml, attn_cnt, chain_flags;
     size_t total;
 };
@@ -95,6 +97,7 @@ Layout make_layout(const pass_config& c) {
         L.sumsq_b = cv.take((d / 128 + 1) * R * 4);
         L.partial_ws = cv.take((size_t)kMaxOps * kMaxCtas * 2 * R * kTileN * 4);
         L.counters = cv.take(4096 * 4);
+        L.ll_ws = cv.take(kLLRegionBytes * kMaxOps);
         const size_t slices = 2 * kMaxCtas + B * c.n_heads;     // upper bound of B * heads * n_split
         L.attn_po = cv.take(slices * 32 * c.d_head * 4);
         L.attn_pml = cv.take(slices * 32 * 2 * 4);
@@ -129,6 +132,7 @@ struct pass_ctx {
     // tensor-core path (bf16 models)
     __nv_bfloat16 *d_xn_bf = nullptr, *d_attn_bf = nullptr, *d_act_bf = nullptr;
     float *d_q_out = nullptr, *d_sumsq_a = nullptr, *d_sumsq_b = nullptr, *d_partial = nullptr;
+    float* d_ll = nullptr;             // hand-over slots of the <=16-row GEMMs, all bits set when idle
     int* d_counters = nullptr;
     float *d_attn_po = nullptr, *d_attn_pml = nullptr;
     int* d_attn_cnt = nullptr;
@@ -285,6 +289,7 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     p.epi = epi;
     p.n_out = n_out;
     p.partial_ws = c->d_partial;
+    p.ll_ws = c->d_ll;
     p.tile_counters = c->d_counters;
     p.status = c->d_status;
     p.eps = c->md.eps;
@@ -325,6 +330,7 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     for (int j = 0; j < n_ops; j++) {
         if (ops[j].p.partial_ws == c->d_partial) {
             ops[j].p.partial_ws = c->d_partial + (size_t)j * region;
+            ops[j].p.ll_ws = c->d_ll + (size_t)j * (kLLRegionBytes / 4);
             ops[j].p.tile_counters = c->d_counters + j * 1024;
         }
         cp.op[j] = ops[j].p;
@@ -693,6 +699,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_sumsq_a = (float*)(w + L.sumsq_a);
         c->d_sumsq_b = (float*)(w + L.sumsq_b);
         c->d_partial = (float*)(w + L.partial_ws);
+        c->d_ll = (float*)(w + L.ll_ws);
         c->d_counters = (int*)(w + L.counters);
         c->d_attn_po = (float*)(w + L.attn_po);
         c->d_attn_pml = (float*)(w + L.attn_pml);
@@ -723,6 +730,9 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.xn_bf, 0, L.total - L.xn_bf, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    // the hand-over slots of the <=16-row GEMMs are EMPTY (all bits set) whenever no launch is using them
+    if (cfg->dtype == PASS_DTYPE_BF16 &&
+        cudaMemsetAsync(w + L.ll_ws, 0xFF, kLLRegionBytes * kMaxOps, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     std::vector<double> inv(cfg->d_head / 2);
     for (int i = 0; i < cfg->d_head / 2; i++)
         inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
@@ -934,6 +944,8 @@ int pass_step_collect(pass_ctx* c, int32_t* out_tokens, int32_t* n_out) {
     const int status = *c->pin_status;
     if (status != 0) {
         CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream));
+        if ((status & kStatusTimeout) && c->d_ll)       // an abandoned launch may have left words in the slots
+            CUDA_TRY(cudaMemsetAsync(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps, c->stream));
         CUDA_TRY(cudaStreamSynchronize(c->stream));
         if (status & kStatusTimeout) return PASS_ERR_TIMEOUT;
         if (status & kStatusNonFinite) return PASS_ERR_NONFINITE;
@@ -1128,6 +1140,7 @@ static int debug_status(pass_ctx* c) {
     CUDA_TRY(cudaMemcpy(&status, c->d_status, 4, cudaMemcpyDeviceToHost));
     if (status) {
         CUDA_TRY(cudaMemset(c->d_status, 0, 4));
+        if ((status & kStatusTimeout) && c->d_ll) CUDA_TRY(cudaMemset(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps));
         return (status & kStatusTimeout) ? PASS_ERR_TIMEOUT : PASS_ERR_STATE;
     }
     return PASS_OK;
@@ -1224,6 +1237,8 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     if (!g_static_scratch_addr[dev]) {          // first call on this device
         void* ptr = nullptr;
         CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        // the hand-over slots start out EMPTY (all bits set); every call leaves them that way
+        CUDA_TRY(cudaMemsetAsync(ptr, 0xFF, kStaticPartialBytes, c->stream));
         g_static_scratch_addr[dev] = ptr;
     }
     char* scratch = (char*)g_static_scratch_addr[dev];
@@ -1254,7 +1269,8 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
     p.logits = y_device;
-    p.partial_ws = (float*)scratch;
+    p.partial_ws = (float*)scratch;          // never used with <= 16 rows
+    p.ll_ws = (float*)scratch;
     p.tile_counters = (int*)(scratch + kStaticPartialBytes);
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
     CUDA_TRY(cudaGetLastError());
