@@ -276,7 +276,8 @@ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int
 }
 
 // ------------------------------------------------------------------------------------ epilogues
-// Thread = one feature of the tile (TMEM lane); v[j] = result for token rows c0 .. c0+7.
+// Thread = one feature of the tile (TMEM lane); v[j] = result for token rows c0 .. c0+NR-1 (NR = 8, or 9 so
+// that the 1 + 2k rows of k = 4 look-ahead tokens go through in one pass).
 struct EpiCtx {
     int lane_in_tile;        // 0..127
     float* s_rstd;           // [kMaxRows]
@@ -294,7 +295,8 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 // loaded (so that this trip to L2 overlaps with another); nullptr = load them here.
 // g_pre / cs_pre: likewise the next norm's gain for this feature (kEpiResid) and the eight rotation pairs
 // (kEpiQKV), fetched by the caller while it was still waiting for the accumulator.
-__device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[8],
+template <int NR>
+__device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[NR],
                                           const float* hv_pre = nullptr, const float* g_pre = nullptr,
                                           const float2* cs_pre = nullptr) {
     const int L = ec.lane_in_tile;
@@ -302,7 +304,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int n = tile * kTileN + L;
         if (n < p.n_out) {
 #pragma unroll
-            for (int j = 0; j < 8; j++)
+            for (int j = 0; j < NR; j++)
                 if (c0 + j < p.R) p.logits[(size_t)(c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
         }
     } else if (p.epi == kEpiQKV) {
@@ -310,17 +312,17 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int n = tile * kTileN + L;
         const int which = n / d, c = n % d, head = c / dh, i = c % dh;
         // everything that is read is fetched before the first store, so that the loads overlap
-        int rs[8], rp[8];
-        float2 cs[8];
+        int rs[NR], rp[NR];
+        float2 cs[NR];
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
+        for (int j = 0; j < NR; j++) {
             const int r = min(c0 + j, p.R - 1);
             rs[j] = ec.s_rseq[r];
             rp[j] = ec.s_rpos[r];
             cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
         }
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
+        for (int j = 0; j < NR; j++) {
             const int r = c0 + j;
             const float x = v[j] * (r < p.R ? ec.s_rstd[r] : 0.f);
             const float other = __shfl_xor_sync(0xffffffffu, x, 1);
@@ -339,12 +341,12 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int n = tile * kTileN + L;
         const float g = g_pre ? *g_pre : (n < d ? __bfloat162float(p.gain_next[n]) : 0.f);
         const int warp_q = (threadIdx.x >> 5) & 3, lane = threadIdx.x & 31;
-        float ss[8], hv[8];
+        float ss[NR], hv[NR];
 #pragma unroll
-        for (int j = 0; j < 8; j++)      // all loads first: they are independent of the stores below
+        for (int j = 0; j < NR; j++)      // all loads first: they are independent of the stores below
             hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < p.R && n < d) ? __ldcg(p.h + (size_t)(c0 + j) * d + n) : 0.f);
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
+        for (int j = 0; j < NR; j++) {
             const int r = c0 + j;
             float hn = 0.f;
             if (r < p.R && n < d) {
@@ -357,32 +359,32 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             }
             ss[j] = hn * hn;
         }
-        // eight butterfly reductions side by side: each level issues eight independent shuffles, so the
-        // shuffle latency is paid five times, not forty
+        // the butterfly reductions of all rows side by side: each level issues NR independent shuffles, so
+        // the shuffle latency is paid five times, not 5 NR times
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-            for (int j = 0; j < 8; j++) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], o);
+            for (int j = 0; j < NR; j++) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], o);
         }
         epi_bar();                                  // s_x free
         if (lane == 0) {
 #pragma unroll
-            for (int j = 0; j < 8; j++) ec.s_x[warp_q * 8 + j] = ss[j];
+            for (int j = 0; j < NR; j++) ec.s_x[warp_q * NR + j] = ss[j];
         }
         epi_bar();
-        if (L < 8 && c0 + L < p.R)
+        if (L < NR && c0 + L < p.R)
             p.sumsq_out[(size_t)tile * kMaxRows + c0 + L] =
-                ec.s_x[L] + ec.s_x[8 + L] + ec.s_x[16 + L] + ec.s_x[24 + L];
+                ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
     } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
         epi_bar();                                  // s_x free
 #pragma unroll
-        for (int j = 0; j < 8; j++) ec.s_x[L * 9 + j] = v[j];
+        for (int j = 0; j < NR; j++) ec.s_x[L * 9 + j] = v[j];
         epi_bar();
         if (L < 64) {
             const int n = tile * 64 + L;
             if (n < p.n_out) {
 #pragma unroll
-                for (int j = 0; j < 8; j++) {
+                for (int j = 0; j < NR; j++) {
                     const int r = c0 + j;
                     if (r < p.R) {
                         const float rs = ec.s_rstd[r];
@@ -806,7 +808,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
                 float2 cs_pre[16] = {};
-                const bool pre = p.rh == 16 && pc.n_pieces > 1 && pc.index == 0;
+                const bool pre = p.rh == 16 && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
@@ -824,7 +826,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 if (et == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
                 const bool whole = pc.n_pieces == 1;
-                const bool ll = p.rh == 16 && !whole;          // counter-free hand-over of the partial sums, fixed finisher
+                const bool ll = p.rh == 16;                    // up to 16 rows: counter-free hand-over, fixed finisher
                 float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
                 int ll_n = 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
@@ -843,61 +845,46 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
-                    if (pc.index != 0) {
+                    if (!whole && pc.index != 0) {
                         // a later part of the tile: hand it to the CTA that holds the tile's first k-blocks
                         float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
 #pragma unroll
                         for (int j = 0; j < 16; j++)
                             if (j < p.R) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
                     } else {
-                        // The tile's first part is this CTA's LAST piece of the GEMM (its range ends inside the
-                        // tile), so it is the natural finisher: the other parts were either computed at the very
-                        // start of their CTAs' ranges or finish together with this one.
+                        // A whole tile, or the tile's first part.  The first part is this CTA's LAST piece of the
+                        // GEMM (its range ends inside the tile), so it is the natural finisher: the other parts
+                        // were either computed at the very start of their CTAs' ranges or finish together with it.
                         tile_done = true;
                         const int n = pc.tile * kTileN + ec.lane_in_tile;
-                        float hv[2][8] = {};
-                        if (p.epi == kEpiResid) {
+                        float hv[16];
 #pragma unroll
-                            for (int j = 0; j < 16; j++)
-                                hv[j >> 3][j & 7] = (j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
-                        }
+                        for (int j = 0; j < 16; j++)
+                            hv[j] = (p.epi == kEpiResid && j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
                         // every contributor but the first keeps its part in slot 0 (its range begins inside the tile)
                         float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
                         const size_t peer_stride = 2 * slot_floats;
-                        float acc9[kLLRows];
-#pragma unroll
-                        for (int j = 0; j < kLLRows; j++) acc9[j] = av[j];
-                        ll_gather(peer, peer_stride, pc.n_pieces - 1, 0, min(p.R, kLLRows), acc9, &s_abort, cp.status);
-                        if (et == 0) PASS_TRACE(oi, 5);
-                        // both halves run through ONE copy of the epilogue code (the loop is kept rolled)
+                        // rows go through the epilogue nine at a time (ONE rolled copy of its code): the 1 + 2k rows
+                        // of up to four look-ahead tokens take a single pass
 #pragma unroll 1
-                        for (int half = 0; half < 2; half++) {
-                            if (half * 8 >= p.R) break;
-                            float a8[8], h8[8];
-                            float2 cs8[8];
-                            if (half == 0) {
+                        for (int c0 = 0; c0 < 16; c0 += kLLRows) {
+                            if (c0 >= p.R) break;
+                            float a9[kLLRows], h9[kLLRows];
+                            float2 cs9[kLLRows];
 #pragma unroll
-                                for (int j = 0; j < 8; j++) a8[j] = acc9[j];
-                            } else {
-                                float rest[kLLRows];
-#pragma unroll
-                                for (int j = 0; j < kLLRows; j++) rest[j] = j < 7 ? av[9 + j] : 0.f;
-                                if (p.R > kLLRows)
-                                    ll_gather(peer, peer_stride, pc.n_pieces - 1, kLLRows, p.R - kLLRows, rest, &s_abort, cp.status);
-                                a8[0] = acc9[8];
-#pragma unroll
-                                for (int j = 1; j < 8; j++) a8[j] = rest[j - 1];
+                            for (int j = 0; j < kLLRows; j++) {
+                                // (row 16 and 17 of the second pass do not exist)
+                                a9[j] = c0 == 0 ? av[j] : (j < 16 - kLLRows ? av[kLLRows + j] : 0.f);
+                                h9[j] = c0 == 0 ? hv[j] : (j < 16 - kLLRows ? hv[kLLRows + j] : 0.f);
+                                cs9[j] = c0 == 0 ? cs_pre[j] : (j < 16 - kLLRows ? cs_pre[kLLRows + j] : make_float2(0.f, 0.f));
                             }
-#pragma unroll
-                            for (int j = 0; j < 8; j++) {
-                                h8[j] = half ? hv[1][j] : hv[0][j];
-                                cs8[j] = half ? cs_pre[8 + j] : cs_pre[j];
-                            }
-                            epi_store(p, ec, pc.tile, half * 8, a8, p.epi == kEpiResid ? h8 : nullptr,
-                                      p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs8 : nullptr);
+                            if (!whole)
+                                ll_gather(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
+                            if (et == 0 && c0 == 0 && !whole) PASS_TRACE(oi, 5);
+                            epi_store<kLLRows>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
+                                               p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs9 : nullptr);
                         }
-                        ll_peer = peer;
-                        ll_n = pc.n_pieces - 1;
+                        if (!whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
                     }
                 } else {
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
@@ -909,7 +896,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
 #pragma unroll
                     for (int j = 0; j < 8; j++) hi[j] += lo[j];
                     if (whole) {
-                        epi_store(p, ec, pc.tile, c0, hi);
+                        epi_store<8>(p, ec, pc.tile, c0, hi);
                     } else {
                         // partial slot layout [rh/4][feature] of float4 (four token rows of one feature): a warp
                         // stores and loads 512 contiguous bytes per instruction
@@ -967,7 +954,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                                     }
                                 }
                             }
-                            epi_store(p, ec, pc.tile, c0, acc);
+                            epi_store<8>(p, ec, pc.tile, c0, acc);
                         }
                     }
                 }
