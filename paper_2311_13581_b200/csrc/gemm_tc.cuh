@@ -479,6 +479,8 @@ struct ChainParams {
     int stages;
     int npad;                  // row padding, shared by all GEMMs of the chain
     int pf_units;              // stages per GEMM that are pulled into L2 while the CTA waits for the previous GEMM
+    int test_stuck;            // test hook: the first GEMM's contributors keep their partial sums to themselves, so
+                               // the finishers' bounded waits run out and the launch reports kStatusTimeout
     int hold;                  // 1: no weight request for a GEMM before this CTA's epilogue of the previous one is over
                                // (helped by 0.02 ms while the hand-over still went through an arrival counter and
                                // costs 0.02 ms since it does not: off by default)
@@ -851,7 +853,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
 #pragma unroll
                         for (int j = 0; j < 16; j++)
-                            if (j < p.R) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
+                            if (j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
                     } else {
                         // A whole tile, or the tile's first part.  The first part is this CTA's LAST piece of the
                         // GEMM (its range ends inside the tile), so it is the natural finisher: the other parts

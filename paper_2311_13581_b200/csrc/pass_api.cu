@@ -316,6 +316,7 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     cp.npad = ops[0].p.npad;
     cp.pf_units = 0;
     cp.pf_units0 = 0;
+    cp.test_stuck = getenv("PASS_GEMM_TEST_STUCK") ? 1 : 0;
     cp.hold = getenv("PASS_GEMM_HOLD") ? atoi(getenv("PASS_GEMM_HOLD")) : 0;
     if (const char* e = getenv("PASS_GEMM_PF")) cp.pf_units = std::max(0, std::min(512, atoi(e)));
     if (const char* e = getenv("PASS_GEMM_PF0")) cp.pf_units0 = std::max(0, std::min(512, atoi(e)));

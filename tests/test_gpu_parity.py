@@ -242,6 +242,39 @@ def test_unk_lookahead_baseline_runs_through_the_same_path():
     ctx.close()
 
 
+# ------------------------------------------------------------------ a wait that runs out
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(monkeypatch):
+    """Every device-side wait has a limit.  The hook makes the contributors of the first GEMM of each
+    launch keep their partial sums to themselves, so the CTAs that finish those tiles wait for words that
+    never come: after the limit (0.2 s) they give up, the other roles follow, the step reports TIMEOUT,
+    the sequence state is untouched, and the next steps are correct again."""
+    import paper_2311_13581_b200 as pb
+    from parity_util import lockstep
+    monkeypatch.setenv("PASS_NO_GRAPH", "1")          # the hook is read when a launch is built
+    shape = SEVENB_2L
+    w = si.make_weights(shape, seed=0, device="cuda:0")
+    w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
+    ctx_len, cap = 512, 600
+    ctx = pb.PassContext(shape, w, 1, cap)
+    be = po.TransformerBackend(shape, w_cpu, cap)
+    _load_synthetic_cache(ctx, [be], shape, ctx_len)
+    ctx.set_state(0, ctx_len, 11)
+    orc = po.PassOracle.__new__(po.PassOracle)
+    orc.be, orc.len, orc.pending, orc.drafts = be, ctx_len, 11, []
+    orc.Q_dft, orc.k_prev, orc.T_prev, orc.last_logits = np.zeros((0, shape.vocab)), None, None, None
+    stats, _ = lockstep(ctx, [orc], 4, 0.0, 2)
+    len_before = ctx.get_debug(pb.PASS_DBG_KV_LEN).copy()
+    monkeypatch.setenv("PASS_GEMM_TEST_STUCK", "1")
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(4, 0.0, None)
+    assert "timed out" in str(e.value)
+    monkeypatch.delenv("PASS_GEMM_TEST_STUCK")
+    assert (ctx.get_debug(pb.PASS_DBG_KV_LEN) == len_before).all()
+    stats, _ = lockstep(ctx, [orc], 4, 0.0, 2, step0=2)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    ctx.close()
+
+
 # ------------------------------------------------------------------ errors never fault
 def test_error_paths(tiny_w):
     pb = _pb()
