@@ -12,9 +12,12 @@
 //     16s, not to 64/128.  Activations are carried as bf16 hi + bf16 lo rows (x = hi + lo), which
 //     doubles N at no HBM cost and keeps activation rounding out of the result.
 //   * stream-K: the (tile, k-block) units of one GEMM are cut into equal contiguous ranges, one per
-//     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is.
-//     A tile cut across CTAs is reduced by the LAST CTA to arrive (counter per tile), which sums
-//     the partials in k order - deterministic - and runs the fused epilogue.
+//     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is; with at
+//     least as many tiles as CTAs only the n_tiles mod CTAs odd tiles are streamed and the GEMM ends
+//     on whole tiles (see get_piece).  A tile cut across CTAs is summed in k order - deterministic -
+//     by one CTA, which then runs the fused epilogue: up to 16 token rows by the CTA holding the
+//     tile's first k-blocks, which finds the other parts in EMPTY-or-value words (no counter, see
+//     ll_gather); more rows by the LAST CTA to arrive (counter per tile).
 //   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 1 TMEM allocation + MMA issue,
 //     warps 2-5 epilogue (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue
 //     of one piece overlaps the main loop of the next.
@@ -50,9 +53,6 @@ struct GemmParams {
     int stages;
     int epi;
     int n_out;                     // output features in total
-    const void* w_base[3];         // the weight matrices behind maps 0..2 (for L2 prefetch), [w_rows][w_ld] bf16
-    int w_rows[3];
-    int w_ld;
     float* partial_ws;             // [gridDim][2][rh][128] fp32: more than 16 rows (arrival counter per tile)
     float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: up to 16 rows
     int* tile_counters;            // [n_tiles], zero between launches
@@ -133,10 +133,6 @@ __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
-}
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
-                 ::"l"((uint64_t)map), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
@@ -478,13 +474,11 @@ struct ChainParams {
     int n_ops;
     int stages;
     int npad;                  // row padding, shared by all GEMMs of the chain
-    int pf_units;              // stages per GEMM that are pulled into L2 while the CTA waits for the previous GEMM
     int test_stuck;            // test hook: the first GEMM's contributors keep their partial sums to themselves, so
                                // the finishers' bounded waits run out and the launch reports kStatusTimeout
     int hold;                  // 1: no weight request for a GEMM before this CTA's epilogue of the previous one is over
                                // (helped by 0.02 ms while the hand-over still went through an arrival counter and
                                // costs 0.02 ms since it does not: off by default)
-    int pf_units0;             // the same for the first GEMM of the launch (waits for the previous kernel)
     int* op_done;              // [kMaxOps] tiles completed per GEMM; zero between launches
     int* ctas_done;            // CTAs that have left the kernel (the last one clears op_done)
     int* status;
@@ -535,7 +529,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_abort;
     __shared__ int s_issued, s_issued_b;
     __shared__ int s_epi_done;
-    __shared__ int s_mma_done;             // last GEMM of the chain whose MMAs this CTA has all issued (-1: none)
     __shared__ int s_last;
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
@@ -579,7 +572,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         s_abort = 0;
         s_issued = 0;
         s_issued_b = 0;
-        s_mma_done = -1;
         s_epi_done = -1;
         s_epi_fail = 0;
         fence_barrier_init();
@@ -669,57 +661,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 }
             }
         }
-    } else if (warp == 7) {
-        // ---------------------------------------------------------------- L2 prefetch (plain loads path)
-        // All 32 lanes walk ahead of the ring (by at most pf_units units) and touch the coming weight
-        // rows with prefetch.global.L2: one 128-byte row segment per lane and instruction.  These go
-        // through the load/store path, not through the TMA queue, so they never sit in front of the
-        // ring's own requests; they keep HBM streaming while the consumers wait for an earlier GEMM.
-        if (cp.pf_units > 0 || cp.pf_units0 > 0) {
-            // One burst per GEMM: when this CTA has issued the last MMA of the previous GEMM, its ring
-            // already holds the first stages of the next one and nothing more can be requested until the
-            // previous GEMM's results exist everywhere.  HBM would idle through that hand-over; instead
-            // the stages that follow the ring's are pulled into L2 now.  Nothing is prefetched while
-            // the previous GEMM still streams (that would only delay the data it is waiting for).
-            int count = 0;
-            Piece pc;
-            bool stop = false;
-            for (int oi = 0; !stop && oi < cp.n_ops; oi++) {
-                const GemmParams& p = cp.op[oi];
-                const int burst = oi == 0 ? cp.pf_units0 : cp.pf_units;
-                int in_op = 0;
-                for (int it = 0; !stop && fetch_piece(oi, it, pc); it++) {
-                    // rows of the tile: plain = 128 rows of one matrix; interleaved = 64 rows of two
-                    const char* base0; const char* base1; int row0, nrows0, nrows1;
-                    if (p.interleave) {
-                        base0 = (const char*)p.w_base[0]; base1 = (const char*)p.w_base[1];
-                        row0 = pc.tile * 64; nrows0 = nrows1 = min(64, p.w_rows[0] - row0);
-                    } else {
-                        int tl = pc.tile, seg = 0;
-                        if (tl >= p.seg_tiles0) { tl -= p.seg_tiles0; seg = 1; if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; seg = 2; } }
-                        base0 = (const char*)p.w_base[seg]; base1 = nullptr;
-                        row0 = tl * kTileN; nrows0 = min(kTileN, p.w_rows[seg] - row0); nrows1 = 0;
-                    }
-                    const size_t ldb = (size_t)p.w_ld * 2;
-                    for (int kb = pc.kb0; kb < pc.kb1 && !stop; kb++, count++, in_op++) {
-                        if (in_op < S || in_op >= S + burst) continue;      // the ring's own / beyond the burst
-                        const long long t0 = clock64();
-                        while (*(volatile int*)&s_mma_done < oi - 1) {
-                            if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { stop = true; break; }
-                            __nanosleep(200);
-                        }
-                        if (stop) break;
-                        if (count < *(volatile int*)&s_issued) continue;    // the ring got there first
-                        const size_t col = (size_t)kb * kBlockK * 2;
-                        if ((kb + 1) * kBlockK > p.w_ld) continue;          // ragged last k-block: leave it to TMA
-                        for (int r = lane; r < nrows0; r += 32)
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base0 + (size_t)(row0 + r) * ldb + col));
-                        for (int r = lane; r < nrows1; r += 32)
-                            asm volatile("prefetch.global.L2 [%0];" ::"l"(base1 + (size_t)(row0 + r) * ldb + col));
-                    }
-                }
-            }
-        }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issue
         if (lane == 0) {
@@ -750,7 +691,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     }
                     if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
                 }
-                *(volatile int*)&s_mma_done = oi;
                 PASS_TRACE(oi, 2);
             }
         }

@@ -314,14 +314,8 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     cp.n_ops = n_ops;
     cp.stages = ops[0].p.stages;
     cp.npad = ops[0].p.npad;
-    cp.pf_units = 0;
-    cp.pf_units0 = 0;
     cp.test_stuck = getenv("PASS_GEMM_TEST_STUCK") ? 1 : 0;
     cp.hold = getenv("PASS_GEMM_HOLD") ? atoi(getenv("PASS_GEMM_HOLD")) : 0;
-    if (const char* e = getenv("PASS_GEMM_PF")) cp.pf_units = std::max(0, std::min(512, atoi(e)));
-    if (const char* e = getenv("PASS_GEMM_PF0")) cp.pf_units0 = std::max(0, std::min(512, atoi(e)));
-    for (int j = 0; j < n_ops; j++)
-        if (!ops[j].p.w_base[0]) cp.pf_units = cp.pf_units0 = 0;      // no raw weight pointers given: nothing to prefetch
     cp.op_done = c->d_chain_flags;
     cp.ctas_done = c->d_chain_flags + kMaxOps;
     cp.status = c->d_status;
@@ -442,11 +436,6 @@ static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
 }
 
 // GEMMs of the decoder layers as chain entries.
-static void fill_weights(GemmParams& p, const void* w0, const void* w1, const void* w2, int rows, int ld) {
-    p.w_base[0] = w0; p.w_base[1] = w1; p.w_base[2] = w2;
-    p.w_rows[0] = p.w_rows[1] = p.w_rows[2] = rows;
-    p.w_ld = ld;
-}
 static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l) {
     typedef __nv_bfloat16 bf;
     const int d = c->md.d, dt = d / kTileN;
@@ -456,7 +445,6 @@ static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, i
     o.p.sumsq_in = c->d_sumsq_a; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
     o.p.q_out = c->d_q_out; o.p.rope_cs = c->d_cs; o.p.row_seq = c->d_row_seq; o.p.row_pos = c->d_row_pos;
     o.p.layer = l; o.p.kc = (bf*)c->kv_k; o.p.vc = (bf*)c->kv_v;
-    fill_weights(o.p, c->wq[l], c->wk[l], c->wv[l], d, d);
     o.a0 = c->tm_wq[l]; o.a1 = c->tm_wk[l]; o.a2 = c->tm_wv[l]; o.b = bm->xn;
     return o;
 }
@@ -471,7 +459,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         ChainOp& o = ch[n++];
         o.p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
         o.p.h = c->d_h; o.p.gain_next = (const bf*)c->norm_ffn[l]; o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_b;
-        fill_weights(o.p, c->wo[l], c->wo[l], c->wo[l], d, d);
         o.a0 = o.a1 = o.a2 = c->tm_wo[l]; o.b = bm->attn;
     }
     {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
@@ -480,7 +467,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p.interleave = 1;
         o.p.sumsq_in = c->d_sumsq_b; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
         o.p.act_out = c->d_act_bf;
-        fill_weights(o.p, c->wg[l], c->wu[l], c->wu[l], f, d);
         o.a0 = c->tm_wg[l]; o.a1 = o.a2 = c->tm_wu[l]; o.b = bm->xn;
     }
     {   // down projection + residual; prepares the input of the next norm
@@ -489,7 +475,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p.h = c->d_h;
         o.p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
         o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_a;
-        fill_weights(o.p, c->wd[l], c->wd[l], c->wd[l], d, f);
         o.a0 = o.a1 = o.a2 = c->tm_wd[l]; o.b = bm->act;
     }
     if (l + 1 < md.n_layers) {
@@ -499,7 +484,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
         o.p.sumsq_in = c->d_sumsq_a; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
         o.p.logits = c->d_logits;
-        fill_weights(o.p, c->lm_head, c->lm_head, c->lm_head, md.V, d);
         o.a0 = o.a1 = o.a2 = c->tm_lm; o.b = bm->xn;
     }
     return n;
