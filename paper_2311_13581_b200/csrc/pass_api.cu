@@ -138,6 +138,8 @@ struct pass_ctx {
     int* d_attn_cnt = nullptr;
     int n_sms = 148;
     bool use_pdl = true;
+    bool attn_long = false;       // this step's contexts are long: twice as many attention slices (see step_launch)
+    int attn_long_from = 3072;    // PASS_ATTN_LONG_FROM: cached positions from which a step counts as long
     bool attn_cluster = true;     // PASS_ATTN_NO_CLUSTER: merge attention slices through global memory
     int attn_debug_stale = 0;     // PASS_ATTN_STALE=n: attention's early part works from a cache length n short
     bool use_tc = false;
@@ -516,6 +518,9 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
             ap.layer = l; ap.kc = (const bf*)c->kv_k; ap.vc = (const bf*)c->kv_v; ap.M = M;
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
+            // Long contexts: the key loop (tensor-core work of 4 warps) outweighs everything that one CTA per
+            // SM buys at short contexts, so the slices are doubled - two CTAs per SM, 8 warps on the keys.
+            if (c->attn_long && ap.n_split * 2 <= 8) ap.n_split *= 2;
             ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
             ap.out = c->d_attn_bf; ap.lo_row0 = rh; ap.debug_stale = c->attn_debug_stale;
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
@@ -693,6 +698,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         c->attn_cluster = getenv("PASS_ATTN_NO_CLUSTER") == nullptr;
+        if (const char* e = getenv("PASS_ATTN_LONG_FROM")) c->attn_long_from = std::max(0, atoi(e));
         if (const char* e = getenv("PASS_ATTN_STALE")) c->attn_debug_stale = std::max(0, atoi(e));
         c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
@@ -879,8 +885,12 @@ static int step_launch(pass_ctx* c, int k, float T) {
     }
     c->have_last = true; c->last_k = k; c->last_T = T; c->last_top_k = c->top_k;
     c->launches = 0;
+    // one graph per (k, short / long contexts): the number of attention slices is part of the launch shape
+    c->attn_long = false;
+    for (int b = 0; b < c->md.B; b++) c->attn_long |= c->len_ub[b] >= c->attn_long_from;
+    const int gkey = k + (c->attn_long ? 1000 : 0);
     if (c->use_graph) {
-        auto it = c->graphs.find(k);
+        auto it = c->graphs.find(gkey);
         if (it == c->graphs.end()) {
             cudaGraph_t g = nullptr;
             CUDA_TRY(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
@@ -891,12 +901,12 @@ static int step_launch(pass_ctx* c, int k, float T) {
             e = cudaGraphInstantiate(&ge, g, 0);
             cudaGraphDestroy(g);
             if (e != cudaSuccess) return PASS_ERR_CUDA;
-            c->graphs[k] = ge;
-            c->graph_launches[k] = c->launches;
-            it = c->graphs.find(k);
+            c->graphs[gkey] = ge;
+            c->graph_launches[gkey] = c->launches;
+            it = c->graphs.find(gkey);
         }
         CUDA_TRY(cudaGraphLaunch(it->second, c->stream));
-        c->last_step_launches = c->graph_launches[k];
+        c->last_step_launches = c->graph_launches[gkey];
     } else {
         enqueue_step_any(c, k);
         CUDA_TRY(cudaGetLastError());
