@@ -240,6 +240,18 @@ int pass_debug_linear(pass_ctx *ctx, int which, int layer, const float *x_device
                       float *y_device);
 
 /*
+ * The work schedule of the weight-streaming GEMM, evaluated on the host (no context, no device):
+ * the `it`-th piece of CTA `cta` out of `n_ctas` for a GEMM of n_tiles output tiles with
+ * kb_per_tile k-blocks each.  Returns 1 and fills out[7] = {tile, kb0, kb1, n_pieces, index, slot,
+ * first_slot} (k-blocks [kb0, kb1) of `tile`; n_pieces CTAs share the tile and this is number
+ * `index` of them in k order; slot = which of the CTA's two partial-sum slots the piece uses),
+ * or returns 0 when the CTA has no such piece, or -1 on invalid arguments.  It is the same function
+ * the kernel runs; the tests check on it what the hand-over of partial sums relies on (every
+ * k-block computed exactly once, the CTAs that share a tile are consecutive, ...).
+ */
+int pass_debug_schedule(int n_tiles, int kb_per_tile, int n_ctas, int cta, int it, int32_t *out);
+
+/*
  * Time that kernel: n_launches launches back to back on the context's stream, cycling over the
  * layers so that every launch streams different weights from HBM (CUDA events; one untimed pass
  * over the layers first).  which as above, except 7; which = 9 times the step's dominant launch, the

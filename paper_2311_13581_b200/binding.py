@@ -23,7 +23,7 @@ PASS_MAX_TOP_K = 1024
 
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
            "pass_step", "pass_step_enqueue", "pass_step_collect", "pass_forward_tokens", "pass_reset",
-           "pass_set_top_k", "pass_step_two_call",
+           "pass_set_top_k", "pass_step_two_call", "pass_debug_schedule",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
            "pass_debug_time_linear", "pass_linear_noalloc"]
@@ -75,6 +75,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_forward_tokens.argtypes = [vp, ci, vp, ci, vp, ci]
     lib.pass_reset.argtypes = [vp, ci]
     lib.pass_set_top_k.argtypes = [vp, ci]
+    lib.pass_debug_schedule.argtypes = [ci, ci, ci, ci, ci, vp]
     lib.pass_set_kv.argtypes = [vp, ci, ci, ci, ci, vp, vp]
     lib.pass_get_kv.argtypes = [vp, ci, ci, ci, ci, vp, vp]
     lib.pass_set_state.argtypes = [vp, ci, ci, ctypes.c_int32]

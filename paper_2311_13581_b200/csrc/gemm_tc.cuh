@@ -215,8 +215,8 @@ struct Piece {
     int first_slot;          // slot used by the tile's first contributor (the only one that may have begun earlier)
 };
 
-__device__ __forceinline__ long long unit_start(long long c, long long U, long long G) { return c * U / G; }
-__device__ __forceinline__ int unit_owner(long long x, long long U, long long G) {
+__host__ __device__ __forceinline__ long long unit_start(long long c, long long U, long long G) { return c * U / G; }
+__host__ __device__ __forceinline__ int unit_owner(long long x, long long U, long long G) {
     return (int)(((x + 1) * G - 1) / U);
 }
 
@@ -228,7 +228,7 @@ __device__ __forceinline__ int unit_owner(long long x, long long U, long long G)
 // CTA computes whole tiles of its own.  The GEMM therefore ends on whole tiles, whose epilogue needs no
 // other CTA: no arrival counter and no trip for partial sums on the path to the next GEMM.  With fewer
 // tiles than CTAs everything is streamed.
-__device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
+__host__ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
     const int rounds = p.n_tiles >= G ? p.n_tiles / G : 0;      // whole tiles per CTA
     const int n_sk = p.n_tiles - rounds * G;                     // tiles that are streamed, [0, n_sk)
     const long long U = (long long)n_sk * p.kb_per_tile;

@@ -1273,6 +1273,19 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     return debug_status(c);
 }
 
+int pass_debug_schedule(int n_tiles, int kb_per_tile, int n_ctas, int cta, int it, int32_t* out) {
+    if (n_tiles < 1 || kb_per_tile < 1 || n_ctas < 1 || cta < 0 || cta >= n_ctas || it < 0 || !out) return -1;
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.n_tiles = n_tiles;
+    p.kb_per_tile = kb_per_tile;
+    Piece pc;
+    if (!get_piece(p, cta, n_ctas, it, pc)) return 0;
+    out[0] = pc.tile; out[1] = pc.kb0; out[2] = pc.kb1; out[3] = pc.n_pieces; out[4] = pc.index;
+    out[5] = pc.slot; out[6] = pc.first_slot;
+    return 1;
+}
+
 int pass_last_step_launches(pass_ctx* c) { return c ? c->last_step_launches : 0; }
 void* pass_stream(pass_ctx* c) { return c ? (void*)c->stream : nullptr; }
 
