@@ -280,6 +280,69 @@ k_split_norm_input(const float* __restrict__ h, const __nv_bfloat16* __restrict_
     }
 }
 
+// The three kernels ahead of a decode step's first GEMM in one: row assembly (k_assemble_step), rotary
+// table (k_rope_table) and the first layer's norm input (k_split_norm_input), same arithmetic.  Grid
+// (rows, d / 1024), 256 threads: thread t of chunk c handles columns 1024 c + 256 j + t, j = 0..3, so warps
+// 0-3 (4-7) of pass j cover tile 8 c + 2 j (+ 1) of 128 columns.
+__global__ void __launch_bounds__(256)
+k_step_input(const __nv_bfloat16* __restrict__ tok_emb, const __nv_bfloat16* __restrict__ la_emb,
+             const SeqState* __restrict__ states, const StepParams* __restrict__ sp, int M, int d, int vocab,
+             float* __restrict__ h, int* __restrict__ row_seq, int* __restrict__ row_pos,
+             const double* __restrict__ inv_freq, int half, float2* __restrict__ cs,
+             const __nv_bfloat16* __restrict__ g, __nv_bfloat16* __restrict__ xn, int lo_row0,
+             float* __restrict__ sumsq) {
+    __shared__ float red[4][8];
+    const int r = blockIdx.x, chunk = blockIdx.y, b = r / M, i = r % M;
+    const SeqState& st = states[b];
+    const int k = sp->k;
+    const int m = effective_m(st, sp);
+    const __nv_bfloat16* src;
+    if (i == 0) {
+        src = tok_emb + (size_t)min(max(st.pending, 0), vocab - 1) * d;
+    } else if (i <= m) {
+        src = tok_emb + (size_t)min(max(st.drafts[i - 1], 0), vocab - 1) * d;
+    } else {
+        const int j = (i - m - 1) % max(k, 1);
+        src = la_emb + (size_t)j * d;
+    }
+    float v[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        const int c = chunk * 1024 + j * 256 + threadIdx.x;
+        v[j] = c < d ? __bfloat162float(src[c]) : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        const int c = chunk * 1024 + j * 256 + threadIdx.x;
+        if (c < d) {
+            h[(size_t)r * d + c] = v[j];
+            const float x = v[j] * __bfloat162float(g[c]);
+            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            xn[(size_t)r * d + c] = hi;
+            xn[(size_t)(lo_row0 + r) * d + c] = __float2bfloat16_rn(x - __bfloat162float(hi));
+        }
+        const float ss = warp_sum(v[j] * v[j]);
+        if ((threadIdx.x & 31) == 0) red[j][threadIdx.x >> 5] = ss;
+    }
+    __syncthreads();
+    if (threadIdx.x < 8) {
+        const int j = threadIdx.x >> 1, w0 = (threadIdx.x & 1) * 4, t = chunk * 8 + threadIdx.x;
+        if (t * 128 < d) sumsq[(size_t)t * kMaxRows + r] = red[j][w0] + red[j][w0 + 1] + red[j][w0 + 2] + red[j][w0 + 3];
+    }
+    if (chunk == 0) {
+        const int pos = st.kv_len + i;
+        if (threadIdx.x == 0) {
+            row_seq[r] = b;
+            row_pos[r] = pos;
+        }
+        for (int q = threadIdx.x; q < half; q += blockDim.x) {
+            double sn, cn;
+            sincos((double)pos * inv_freq[q], &sn, &cn);
+            cs[(size_t)r * half + q] = make_float2((float)cn, (float)sn);
+        }
+    }
+}
+
 // Plain split of float32 rows into bf16 hi + lo rows (no gain).
 __global__ void k_split_rows(const float* __restrict__ x, int K, __nv_bfloat16* __restrict__ out, int lo_row0) {
     const int r = blockIdx.y;

@@ -497,14 +497,17 @@ static void launch_ops(pass_ctx* c, ChainOp* ch, int n) {
 }
 
 // R rows = n_seq sequences x M rows each (M = R when n_seq == 1).
-static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head) {
+// input_ready: the rotary table and the first layer's norm input have been produced already (k_step_input).
+static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool input_ready = false) {
     const ModelDims& md = c->md;
     const int d = md.d, npad = npad_for(R), rh = npad / 2;
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     typedef __nv_bfloat16 bf;
-    LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
-    LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
+    if (!input_ready) {
+        LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
+        LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
+    }
     ChainOp chain[kMaxOps];
     // Kernels of a step: QKV_0 | per layer: attention, then ONE launch running
     // O-projection -> gate|up -> down -> (next layer's QKV, or the output head after the last layer).
@@ -575,11 +578,15 @@ template <typename WT>
 static void enqueue_step(pass_ctx* c, int k) {
     const ModelDims& md = c->md;
     const int M = 1 + 2 * k, R = md.B * M;
-    LAUNCH(c, (k_assemble_step<WT>), R, 256, (const WT*)c->tok_emb, (const WT*)c->la_emb, c->d_states,
-           c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos);
     if (c->use_tc) {
-        enqueue_layers_tc(c, R, md.B, true);
+        typedef __nv_bfloat16 bf;
+        LAUNCH(c, k_step_input, dim3(R, (md.d + 1023) / 1024), 256, (const bf*)c->tok_emb, (const bf*)c->la_emb,
+               c->d_states, c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos, c->d_invfreq, md.dh / 2,
+               c->d_cs, (const bf*)c->norm_attn[0], c->d_xn_bf, npad_for(R) / 2, c->d_sumsq_a);
+        enqueue_layers_tc(c, R, md.B, true, true);
     } else {
+        LAUNCH(c, (k_assemble_step<WT>), R, 256, (const WT*)c->tok_emb, (const WT*)c->la_emb, c->d_states,
+               c->d_params, M, md.d, md.V, c->d_h, c->d_row_seq, c->d_row_pos);
         enqueue_layers<WT>(c, R);
         enqueue_head<WT>(c, R);
     }
