@@ -269,17 +269,19 @@ int pass_debug_time_linear(pass_ctx *ctx, int which, int R, int n_launches, floa
  * footprint was fixed up front (a serving process that handed all free HBM to its KV cache and
  * weights), a real-time loop where an allocation could stall or fail, or a host that embeds the
  * library and owns every device byte itself.  The split-K reduction of the GEMM needs scratch
- * (partial sums of output tiles shared by several CTAs, one arrival counter per tile); here that
- * scratch is a fixed array inside the library image, about 2.6 MB that every GPU loading the library
- * holds until the process exits.  The call itself makes no cudaMalloc / cudaFree and calls no
+ * (slots through which CTAs that share an output tile hand their partial sums to the one that
+ * finishes it); here that scratch is a fixed array inside the library image, about 2.6 MB that
+ * every GPU loading the library holds until the process exits.  The call itself makes no cudaMalloc / cudaFree and calls no
  * allocating library routine.  Weights and the activation staging rows are still the context's.
  *
  * Limit: R <= 16 rows.  More rows return PASS_ERR_CAPACITY (nothing runs).
  * First call on a device: looks up the device address of the built-in array (cudaGetSymbolAddress,
- * with that device current) and remembers it; make that first call outside any stream capture.
- * Sharing: all calls, from every context on the device, use the same array.  The arrival counters
- * are cleared at the start of each call; partial sums left by an earlier call are overwritten before
- * they are read.  Two calls that overlap on the GPU (different streams, no ordering) race on it:
+ * with that device current), remembers it and marks every slot empty (a memset on the context's
+ * stream); make that first call outside any stream capture.
+ * Sharing: all calls, from every context on the device, use the same array.  A slot word is either
+ * empty or a partial sum; the CTA that consumes a word marks it empty again, so each call leaves
+ * the array as it found it (after a call that returned PASS_ERR_TIMEOUT the whole array is marked
+ * empty again).  Two calls that overlap on the GPU (different streams, no ordering) race on it:
  * keep them ordered.
  * Arguments, results and the other errors are those of pass_debug_linear.  Synchronises.
  */

@@ -1277,7 +1277,10 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
     CUDA_TRY(cudaGetLastError());
     CUDA_TRY(cudaStreamSynchronize(c->stream));
-    return debug_status(c);
+    const int rc = debug_status(c);
+    if (rc == PASS_ERR_TIMEOUT)     // an abandoned launch may have left words in the shared slots
+        CUDA_TRY(cudaMemset(scratch, 0xFF, kStaticPartialBytes));
+    return rc;
 }
 
 int pass_debug_schedule(int n_tiles, int kb_per_tile, int n_ctas, int cta, int it, int32_t* out) {
