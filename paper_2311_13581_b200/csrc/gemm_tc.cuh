@@ -278,8 +278,7 @@ struct EpiCtx {
     int lane_in_tile;        // 0..127
     float* s_rstd;           // [kMaxRows]
     float* s_x;              // [128][9] exchange buffer
-    const int* s_rseq;       // [kMaxRows] sequence of each token row   (kEpiQKV)
-    const int* s_rpos;       // [kMaxRows] position of each token row   (kEpiQKV)
+    const unsigned long long* s_kvoff;   // [kMaxRows] cache offset of head 0, feature 0 of each token row (kEpiQKV)
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -308,13 +307,13 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const int n = tile * kTileN + L;
         const int which = n / d, c = n % d, head = c / dh, i = c % dh;
         // everything that is read is fetched before the first store, so that the loads overlap
-        int rs[NR], rp[NR];
+        size_t kvo[NR];
         float2 cs[NR];
+        const size_t head_off = ((size_t)head * p.md.cap) * dh + i;
 #pragma unroll
         for (int j = 0; j < NR; j++) {
             const int r = min(c0 + j, p.R - 1);
-            rs[j] = ec.s_rseq[r];
-            rp[j] = ec.s_rpos[r];
+            kvo[j] = (size_t)ec.s_kvoff[r] + head_off;
             cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
         }
 #pragma unroll
@@ -324,11 +323,11 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             const float other = __shfl_xor_sync(0xffffffffu, x, 1);
             if (r < p.R) {
                 if (which == 2) {
-                    p.vc[kv_index(p.md, p.layer, rs[j], head, rp[j]) + i] = __float2bfloat16_rn(x);
+                    p.vc[kvo[j]] = __float2bfloat16_rn(x);
                 } else {
                     const float y = (i & 1) ? other * cs[j].y + x * cs[j].x : x * cs[j].x - other * cs[j].y;
                     if (which == 0) p.q_out[(size_t)r * d + c] = y;
-                    else p.kc[kv_index(p.md, p.layer, rs[j], head, rp[j]) + i] = __float2bfloat16_rn(y);
+                    else p.kc[kvo[j]] = __float2bfloat16_rn(y);
                 }
             }
         }
@@ -532,7 +531,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_last;
     __shared__ int s_epi_fail;
     __shared__ float s_rstd[kMaxRows];
-    __shared__ int s_rseq[kMaxRows], s_rpos[kMaxRows];
+    __shared__ unsigned long long s_kvoff[kMaxRows];
     __shared__ float s_x[128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
@@ -701,8 +700,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         ec.lane_in_tile = wq * 32 + lane;
         ec.s_rstd = s_rstd;
         ec.s_x = s_x;
-        ec.s_rseq = s_rseq;
-        ec.s_rpos = s_rpos;
+        ec.s_kvoff = s_kvoff;
         const int et = (warp - 2) * 32 + lane;        // 0..127
         griddep_wait();
         int pidx = 0;
@@ -739,7 +737,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 ss += __shfl_xor_sync(0xffffffffu, ss, 4);
                 if (r < p.R && l8 == 0) {
                     s_rstd[r] = p.sumsq_in ? rsqrtf(ss * p.inv_d_in + p.eps) : 1.f;
-                    if (p.epi == kEpiQKV) { s_rseq[r] = __ldg(p.row_seq + r); s_rpos[r] = __ldg(p.row_pos + r); }
+                    if (p.epi == kEpiQKV)
+                        s_kvoff[r] = kv_index(p.md, p.layer, __ldg(p.row_seq + r), 0, __ldg(p.row_pos + r));
                 }
             }
             epi_bar();
