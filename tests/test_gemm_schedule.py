@@ -17,6 +17,7 @@ import numpy as np
 import pytest
 
 import paper_2311_13581_b200 as pb
+from paper_2311_13581_b200.build import build_library
 
 
 def pieces(lib, n_tiles, kb, G, cta):
@@ -43,6 +44,7 @@ SHAPES = [
 
 @pytest.mark.parametrize("n_tiles,kb,G", SHAPES)
 def test_schedule_invariants(n_tiles, kb, G):
+    build_library()
     lib = pb.load_library()
     cover = np.zeros((n_tiles, kb), dtype=np.int32)
     by_tile = {}
@@ -90,6 +92,7 @@ def test_schedule_invariants(n_tiles, kb, G):
 
 
 def test_schedule_rejects_bad_arguments():
+    build_library()
     lib = pb.load_library()
     out = (ctypes.c_int32 * 7)()
     assert lib.pass_debug_schedule(0, 4, 8, 0, 0, out) == -1
