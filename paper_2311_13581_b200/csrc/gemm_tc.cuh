@@ -371,24 +371,26 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             p.sumsq_out[(size_t)tile * kMaxRows + c0 + L] =
                 ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
     } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
+        // Both halves of the threads work after the exchange: a gate lane finishes the even rows of its
+        // feature (it reads the up values from the exchange buffer), the matching up lane the odd rows
+        // (it reads the gate values).
         epi_bar();                                  // s_x free
 #pragma unroll
         for (int j = 0; j < NR; j++) ec.s_x[L * 9 + j] = v[j];
         epi_bar();
-        if (L < 64) {
-            const int n = tile * 64 + L;
-            if (n < p.n_out) {
+        const int feat = L & 63, other = L < 64 ? L + 64 : L - 64, n = tile * 64 + feat;
+        if (n < p.n_out) {
 #pragma unroll
-                for (int j = 0; j < NR; j++) {
-                    const int r = c0 + j;
-                    if (r < p.R) {
-                        const float rs = ec.s_rstd[r];
-                        const float g = v[j] * rs, u = ec.s_x[(L + 64) * 9 + j] * rs;
-                        __nv_bfloat16 hi, lo;
-                        split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
-                        p.act_out[(size_t)r * p.n_out + n] = hi;
-                        p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
-                    }
+            for (int j = 0; j < NR; j++) {
+                const int r = c0 + j;
+                if (r < p.R && ((j & 1) == (L >> 6))) {
+                    const float rs = ec.s_rstd[r];
+                    const float mine = v[j] * rs, theirs = ec.s_x[other * 9 + j] * rs;
+                    const float g = L < 64 ? mine : theirs, u = L < 64 ? theirs : mine;
+                    __nv_bfloat16 hi, lo;
+                    split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
+                    p.act_out[(size_t)r * p.n_out + n] = hi;
+                    p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
                 }
             }
         }
