@@ -140,6 +140,21 @@ def test_changing_k_and_temperature_between_steps(tiny_w):
     ctx.close()
 
 
+def test_bf16_changing_k_alternates_between_the_two_partial_sum_protocols():
+    """k = 4, 1, 0 (up to 16 rows: partial sums handed over through EMPTY-or-value words, with 9, 3 and 1
+    live rows) and k = 8 (17 rows: arrival counters) in one context, back and forth: each protocol must
+    find its scratch as it left it, and the graphs of the different k must not disturb each other."""
+    from parity_util import lockstep, make_pair
+    prompt = si.make_prompt(TINY_BF16, 40)
+    ctx, oracles, _ = make_pair(TINY_BF16, 1, 400, [prompt], seed=1)
+    step = 0
+    for k, T in ((4, 0.8), (1, 0.8), (8, 0.8), (0, 0.8), (4, 0.0), (8, 0.0), (2, 0.9), (4, 0.8)):
+        stats, _ = lockstep(ctx, oracles, k, T, 3, step0=step, check_A=False)
+        step += 3
+        assert stats["max_logit_err"] <= 1e-2, (k, T, stats)
+    ctx.close()
+
+
 # ------------------------------------------------------------------ top-k sampling
 @pytest.mark.parametrize("top_k,T", [(10, 0.8), (25, 0.5), (1, 1.0), (3, 0.2)])
 def test_tiny_fp32_top_k_sampling(tiny_w, top_k, T):
