@@ -480,8 +480,9 @@ struct ChainParams {
     int hold;                  // 1: no weight request for a GEMM before this CTA's epilogue of the previous one is over
                                // (helped by 0.02 ms while the hand-over still went through an arrival counter and
                                // costs 0.02 ms since it does not: off by default)
-    int* op_done;              // [kMaxOps] tiles completed per GEMM; zero between launches
-    int* ctas_done;            // CTAs that have left the kernel (the last one clears op_done)
+    int* op_done;              // [kMaxOps] tiles completed by the GEMM in chain position i, counted over ALL launches
+                               // since the counters were last cleared (the host clears them at the start of a forward)
+    int op_target[kMaxOps];    // value of op_done[i] once this launch's GEMM i is complete
     int* status;
     unsigned long long* trace;     // optional %globaltimer stamps [kMaxOps][CTA][8] of this launch (nullptr = off)
     GemmParams op[kMaxOps];
@@ -637,7 +638,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
                 if (oi > 0) {
                     // activations of this GEMM = results of the previous one, written by other SMs
-                    if (!wait_count(cp.op_done + oi - 1, cp.op[oi - 1].n_tiles, &s_abort, cp.status)) break;
+                    if (!wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status)) break;
                     asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
                 }
                 PASS_TRACE(oi, 0);
@@ -712,7 +713,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             const GemmParams& p = cp.op[oi];
             if (oi > 0) {
                 // one thread waits for the previous GEMM; the outcome is made uniform through the barrier
-                if (et == 0 && !wait_count(cp.op_done + oi - 1, cp.op[oi - 1].n_tiles, &s_abort, cp.status))
+                if (et == 0 && !wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status))
                     *(volatile int*)&s_epi_fail = 1;
                 epi_bar();
                 if (*(volatile int*)&s_epi_fail) { ok = false; break; }
@@ -935,15 +936,6 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
-    }
-    if (cp.n_ops > 1 && threadIdx.x == 0) {
-        // the last CTA to leave has seen every CTA pass all of its waits: clear the counters for the next launch
-        int prev;
-        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(cp.ctas_done) : "memory");
-        if (prev == G - 1) {
-            for (int i = 0; i < kMaxOps; i++) cp.op_done[i] = 0;
-            *cp.ctas_done = 0;
-        }
     }
 }
 

@@ -145,6 +145,7 @@ struct pass_ctx {
     bool use_tc = false;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
     int trace_launch = 0;
+    int chain_done_total[kMaxOps] = {0, 0, 0, 0};   // host mirror of what the counters reach (see launch_chain)
     int* d_chain_flags = nullptr;      // [kMaxOps] tiles done per GEMM of a chain, [kMaxOps] = CTAs done               // bf16 models run the GEMMs on tcgen05
     std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
     std::vector<CUtensorMap> tm_wg_plain, tm_wu_plain;   // 128-row boxes, for running gate or up alone
@@ -319,7 +320,12 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     cp.test_stuck = getenv("PASS_GEMM_TEST_STUCK") ? 1 : 0;
     cp.hold = getenv("PASS_GEMM_HOLD") ? atoi(getenv("PASS_GEMM_HOLD")) : 0;
     cp.op_done = c->d_chain_flags;
-    cp.ctas_done = c->d_chain_flags + kMaxOps;
+    for (int j = 0; j < kMaxOps; j++) {
+        // counters only grow between two clears: each launch waits for the totals that include its own tiles,
+        // so nobody has to count the CTAs out and clear them at the end of a launch
+        if (j + 1 < n_ops) c->chain_done_total[j] += ops[j].p.n_tiles;      // the last GEMM of a launch signals nobody
+        cp.op_target[j] = c->chain_done_total[j];
+    }
     cp.status = c->d_status;
     if (c->trace && c->trace_launch < 48)      // the verify scratch (E) doubles as the trace buffer
         cp.trace = (unsigned long long*)c->vb.E + (size_t)(c->trace_launch++) * kMaxOps * kMaxCtas * 8;
@@ -360,6 +366,13 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     cfg.numAttrs = c->use_pdl ? 1 : 0;
     cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, cp);
     c->launches++;
+}
+
+// Start of a forward: the chain's completion counters go back to zero (on the device, in stream order, and
+// in the host's mirror).  Also what makes the next forward right after one that was abandoned on a time-out.
+static void chain_counters_clear(pass_ctx* c) {
+    cudaMemsetAsync(c->d_chain_flags, 0, sizeof(int) * kMaxOps, c->stream);
+    for (int j = 0; j < kMaxOps; j++) c->chain_done_total[j] = 0;
 }
 
 static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
@@ -504,6 +517,7 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     typedef __nv_bfloat16 bf;
+    chain_counters_clear(c);
     if (!input_ready) {
         LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
         LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
@@ -1189,6 +1203,7 @@ int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float*
         }
     };
     if (which == 9) {              // rows at position 0 of sequence 0: the QKV epilogue needs valid row tables
+        chain_counters_clear(c);
         CUDA_TRY(cudaMemsetAsync(c->d_row_seq, 0, sizeof(int) * kMaxRows, c->stream));
         CUDA_TRY(cudaMemsetAsync(c->d_row_pos, 0, sizeof(int) * kMaxRows, c->stream));
     }
