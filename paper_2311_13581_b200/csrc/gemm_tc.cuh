@@ -467,8 +467,10 @@ __device__ __forceinline__ void ll_reset(float* first, size_t stride, int n_othe
 // shared-memory ring stays full of weights while the consumers wait for the previous GEMM's epilogues.
 // The wait itself is a counter per GEMM ("tiles whose epilogue is complete"), bumped with release
 // semantics by the CTA that finishes a tile and read with acquire semantics by every CTA's activation
-// producer and epilogue warps before they touch the next GEMM.  All CTAs of the grid are resident
-// (one per SM), the counter only ever waits for work of an EARLIER GEMM, and every wait is bounded.
+// producer and epilogue warps before they touch the next GEMM.  The counters only grow from launch to
+// launch (the host clears them at the start of a forward and tells each launch which totals to wait for),
+// so a launch ends without any bookkeeping.  All CTAs of the grid are resident (one per SM), the counter
+// only ever waits for work of an EARLIER GEMM, and every wait is bounded.
 constexpr int kMaxOps = 4;
 struct ChainMaps { CUtensorMap m[kMaxOps][4]; };      // per GEMM: weight maps 0..2, activation map
 struct ChainParams {

@@ -146,7 +146,7 @@ struct pass_ctx {
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
     int trace_launch = 0;
     int chain_done_total[kMaxOps] = {0, 0, 0, 0};   // host mirror of what the counters reach (see launch_chain)
-    int* d_chain_flags = nullptr;      // [kMaxOps] tiles done per GEMM of a chain, [kMaxOps] = CTAs done               // bf16 models run the GEMMs on tcgen05
+    int* d_chain_flags = nullptr;      // [kMaxOps] tiles done per GEMM position of a chain, growing until the next clear
     std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
     std::vector<CUtensorMap> tm_wg_plain, tm_wu_plain;   // 128-row boxes, for running gate or up alone
     CUtensorMap tm_lm;
