@@ -35,7 +35,7 @@ CHAIN_TRAFFIC_BYTES = 407476224 + 7009280
 METRIC = "PaSS ms/step and accepted tok/s at 7B-shape bf16 batch 1; HBM GB/s vs 8 TB/s"
 
 WORKLOADS = {
-    # BASELINE configs[1]: the configuration the metric is quoted on
+    # the configuration the headline metric is quoted on
     "7b-k4-ctx512-greedy": dict(shape="7b", k=4, prompt=512, T=0.0, batch=1),
     "7b-k4-ctx2048-T0.8": dict(shape="7b", k=4, prompt=2048, T=0.8, batch=1),
     "7b-k4-ctx8192-T1.0": dict(shape="7b", k=4, prompt=8192, T=1.0, batch=1),
