@@ -397,8 +397,9 @@ class PassOracle:
         P_tgt = np.stack([softmax_T(Z[j], temperature, top_k) for j in range(m + 1)])
         a, y, info = verify(P_tgt, Q_dft, self.drafts, u[:m], u[k])
         info["final_margin"] = invcdf_margin(info["final_law"], u[k])
-        srt = np.sort(Z[a])
-        info["top2_margin"] = float(srt[-1] - srt[-2])
+        # top-2 logit gap of every target row (row j decides draft j+1, row a the final token)
+        info["row_top2"] = [float(np.diff(np.sort(Z[j])[-2:])[0]) for j in range(m + 1)]
+        info["top2_margin"] = info["row_top2"][a]
         info["m"] = m
         dec = {"m": m, "n_accepted": a, "final": y, "emitted": list(self.drafts[:a]) + [y],
                "new_drafts": [], "Qn": np.zeros((0, self.be.vocab)), "info": info}
