@@ -64,8 +64,8 @@ typedef struct {
 
 /* Device pointers to the weights, canonical [out_features, in_features] row-major,
  * all of type cfg.dtype.  Per-layer entries are HOST arrays of n_layers device pointers.
- * la_emb is the [k_max, d_model] look-ahead table ("Look-ahead embeddings":
- * L extra INPUT embeddings; the output dictionary is unchanged). */
+ * la_emb is the [k_max, d_model] look-ahead table (section "Look-ahead embeddings":
+ * extra rows of the INPUT embedding only; the output head keeps the original vocabulary). */
 typedef struct {
     const void *tok_emb;      /* [vocab, d_model] */
     const void *la_emb;       /* [k_max, d_model] */
@@ -101,8 +101,8 @@ int pass_create(const pass_config *cfg, void *kv_k_device, void *kv_v_device, si
 int pass_load_weights(pass_ctx *ctx, const pass_weights *w);
 
 /*
- * Prompt processing for sequence `seq` (Algorithm 1: "initial prompt sequence
- * x_0..x_t; n <- t").  Caches K/V of tokens[0..n-2]; tokens[n-1] becomes the pending
+ * Prompt processing for sequence `seq` (Algorithm 1, its input: the prompt the loop
+ * starts from).  Caches K/V of tokens[0..n-2]; tokens[n-1] becomes the pending
  * token that the first pass_step feeds; pending drafts are dropped.  n >= 1.
  * Resets the sequence first.  Synchronises the stream.
  * Errors: INVALID_ARG (bad seq, n < 1, id outside [0, vocab)), CAPACITY (n-1 > kv_capacity),
@@ -117,7 +117,7 @@ int pass_prefill(pass_ctx *ctx, int seq, const int32_t *tokens, int n);
  *   P_tgt,j = softmax(logits_j / T) for j = 0..m          (validation phase of Algorithm 1)
  *   draft j is accepted iff u[j-1] < min(1, P_tgt,j-1[d_j] / Q_dft,j[d_j])   (strict <)
  *   first rejection at j: final token y ~ norm(max(0, P_tgt,j-1 - Q_dft,j)) and stop;
- *   no rejection:         final token y ~ P_tgt,m  ("sample extra token")
+ *   no rejection:         final token y ~ P_tgt,m  (the bonus token that ends Algorithm 1's loop body)
  *   emitted tokens = accepted drafts then y; len += number emitted; pending = y
  *   if no draft was rejected the k rows after them give the next drafts
  *   d'_t ~ Q'_t = softmax(logits_{m+t} / T) (drafting phase), else the next call has m = 0.
@@ -167,12 +167,15 @@ int pass_step_two_call(pass_ctx *ctx, int L, float temperature, const float *uni
  */
 int pass_step_enqueue(pass_ctx *ctx, int k_lookahead, float temperature,
                       const float *uniforms_device);
-/* Synchronise and fetch the LAST enqueued step's result (same meaning as in pass_step). */
+/* Synchronise and fetch the LAST enqueued step's result (same meaning as in pass_step).
+ * The context keeps one result record per sequence: of several steps enqueued without a collect in
+ * between, only the last one's emitted tokens can be read back (the lengths, pending tokens and
+ * drafts are right for all of them).  Collect after every step whose tokens are wanted. */
 int pass_step_collect(pass_ctx *ctx, int32_t *out_tokens, int32_t *n_out);
 
 /*
- * Multi-token forward for one sequence: n rows appended at positions len .. len+n-1
- * ("a single forward pass on n tokens in parallel").  ids in [0, vocab) are vocabulary
+ * Multi-token forward for one sequence: n rows appended at positions len .. len+n-1, all
+ * scored by one model call (section "Parallel Speculative Sampling").  ids in [0, vocab) are vocabulary
  * tokens; id = vocab + j (0 <= j < k_max) feeds look-ahead embedding j as an input row.
  *   logits_out_device : [n][vocab] float32 on the device, or NULL.
  *   commit            : rows whose K/V are kept, 0..n; len += commit.  Rows after them
@@ -227,8 +230,8 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
 /*
- * One weight-streaming GEMM of the step on its own (bf16 models only): the "forward pass on n
- * tokens" reduced to a single matrix, y[r][n] = sum_k x[r][k] W[n][k] for R <= PASS_MAX_ROWS rows.
+ * One weight-streaming GEMM of the step on its own (bf16 models only): the multi-token model call
+ * reduced to a single matrix, y[r][n] = sum_k x[r][k] W[n][k] for R <= PASS_MAX_ROWS rows.
  *   which : 0 wq, 1 wk, 2 wv, 3 wo, 4 wg, 5 wu, 6 wd (K = d_ffn), 7 lm_head (layer ignored),
  *           8 gate|up as the step reads them: output blocks of 128 = 64 gate then 64 up features,
  *           N = ceil(d_ffn/64)*128.
@@ -269,10 +272,13 @@ int pass_debug_time_linear(pass_ctx *ctx, int which, int R, int n_launches, floa
  * footprint was fixed up front (a serving process that handed all free HBM to its KV cache and
  * weights), a real-time loop where an allocation could stall or fail, or a host that embeds the
  * library and owns every device byte itself.  The split-K reduction of the GEMM needs scratch
- * (slots through which CTAs that share an output tile hand their partial sums to the one that
+ * (words through which CTAs that share an output tile hand their partial sums to the one that
  * finishes it); here that scratch is a fixed array inside the library image, about 2.6 MB that
- * every GPU loading the library holds until the process exits.  The call itself makes no cudaMalloc / cudaFree and calls no
- * allocating library routine.  Weights and the activation staging rows are still the context's.
+ * every GPU loading the library holds until the process exits.  The call itself makes no cudaMalloc /
+ * cudaFree and calls no allocating library routine.  Weights and the activation staging rows are still
+ * the context's.  Every call, whatever R, runs with the rows padded to 16 so that only the
+ * empty-or-value word protocol ever writes to the array (the step's other hand-over protocol, arrival
+ * counters with raw partial sums, would leave non-empty words behind).
  *
  * Limit: R <= 16 rows.  More rows return PASS_ERR_CAPACITY (nothing runs).
  * First call on a device: looks up the device address of the built-in array (cudaGetSymbolAddress,
@@ -287,6 +293,21 @@ int pass_debug_time_linear(pass_ctx *ctx, int which, int R, int n_launches, floa
  */
 int pass_linear_noalloc(pass_ctx *ctx, int which, int layer, const float *x_device, int R,
                         float *y_device);
+
+/*
+ * Switches for the tests of the library's own error handling (no counterpart in the paper).  They are
+ * per context, off by default, and are NOT read from the environment, so that nothing outside the
+ * process can turn them on.  Setting one synchronises and drops the captured step graphs.
+ *   PASS_HOOK_GEMM_STUCK, value 0/1: contributors of the first GEMM of every launch keep their partial
+ *       sums to themselves, so the finishers' bounded waits run out (about 0.2 s) and the call returns
+ *       PASS_ERR_TIMEOUT with the sequence state untouched.
+ *   PASS_HOOK_ATTN_STALE, value n >= 0: the attention kernel's early fetch pretends the cache is n
+ *       positions shorter than it is, which forces its re-check and restart path.
+ * Errors: INVALID_ARG.
+ */
+#define PASS_HOOK_GEMM_STUCK 0
+#define PASS_HOOK_ATTN_STALE 1
+int pass_debug_set(pass_ctx *ctx, int hook, int value);
 
 /* Number of kernel launches (graph nodes) of the last pass_step / pass_step_enqueue. */
 int pass_last_step_launches(pass_ctx *ctx);

@@ -15,9 +15,12 @@
 //     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is; with at
 //     least as many tiles as CTAs only the n_tiles mod CTAs odd tiles are streamed and the GEMM ends
 //     on whole tiles (see get_piece).  A tile cut across CTAs is summed in k order - deterministic -
-//     by one CTA, which then runs the fused epilogue: up to 16 token rows by the CTA holding the
-//     tile's first k-blocks, which finds the other parts in EMPTY-or-value words (no counter, see
-//     ll_gather); more rows by the LAST CTA to arrive (counter per tile).
+//     by one CTA, which then runs the fused epilogue.  Which CTA, and how it learns that the parts
+//     are there, depends on the row padding: with 16 rows per half (npad = 32, i.e. 9 to 16 token
+//     rows: k = 4..7 look-ahead tokens at batch 1) it is the CTA holding the tile's first k-blocks,
+//     which finds the other parts in EMPTY-or-value words (no counter, see ll_gather); with any other
+//     padding (1 to 8 rows: k = 0..3; 17 rows and more: k = 8, batches, prompt chunks) it is the LAST
+//     CTA to arrive (counter per tile).
 //   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 1 TMEM allocation + MMA issue,
 //     warps 2-5 epilogue (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue
 //     of one piece overlaps the main loop of the next.
@@ -53,8 +56,8 @@ struct GemmParams {
     int stages;
     int epi;
     int n_out;                     // output features in total
-    float* partial_ws;             // [gridDim][2][rh][128] fp32: more than 16 rows (arrival counter per tile)
-    float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: up to 16 rows
+    float* partial_ws;             // [gridDim][2][rh][128] fp32: rh != 16 (arrival counter per tile)
+    float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: rh == 16 (9..16 rows)
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
     // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
@@ -397,7 +400,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
     }
 }
 
-// Partial sums of up to 16 token rows are handed over without a counter: a slot word is either EMPTY (all
+// With 16 rows per half (9 to 16 token rows) partial sums are handed over without a counter: a slot word is either EMPTY (all
 // bits set - a NaN pattern that fp32 arithmetic never produces, it makes the canonical 0x7fffffff) or a
 // value.  Contributors just store their values; the finisher loads the words it needs and repeats the
 // load until none of them is empty; when it is done with a tile it stores EMPTY back, so every launch
@@ -477,11 +480,10 @@ struct ChainParams {
     int n_ops;
     int stages;
     int npad;                  // row padding, shared by all GEMMs of the chain
-    int test_stuck;            // test hook: the first GEMM's contributors keep their partial sums to themselves, so
-                               // the finishers' bounded waits run out and the launch reports kStatusTimeout
+    int test_stuck;            // test hook: the first GEMM's contributors keep their partial sums to themselves (or do
+                               // not announce them), so a bounded wait runs out and the launch reports kStatusTimeout
     int hold;                  // 1: no weight request for a GEMM before this CTA's epilogue of the previous one is over
-                               // (helped by 0.02 ms while the hand-over still went through an arrival counter and
-                               // costs 0.02 ms since it does not: off by default)
+                               // (off by default)
     int* op_done;              // [kMaxOps] tiles completed by the GEMM in chain position i, counted over ALL launches
                                // since the counters were last cleared (the host clears them at the start of a forward)
     int op_target[kMaxOps];    // value of op_done[i] once this launch's GEMM i is complete
@@ -773,7 +775,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 if (et == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
                 const bool whole = pc.n_pieces == 1;
-                const bool ll = p.rh == 16;                    // up to 16 rows: counter-free hand-over, fixed finisher
+                const bool ll = p.rh == 16;                    // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
                 float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
                 int ll_n = 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
@@ -856,17 +858,21 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
                 if (!whole) {
-                    // More than 16 rows (prompt chunks): the last CTA to deliver its part of the tile sums all
+                    // Any other padding (1..8 rows, 17 and more): the last CTA to deliver its part of the tile sums all
                     // parts in k order.  The barrier orders every thread's partial stores before thread 0's
                     // acq_rel atomic (release is cumulative), and the loads after the second barrier behind
                     // its acquire.
                     epi_bar();
                     if (et == 0) {
-                        int prev;
-                        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
-                                     : "=r"(prev) : "l"(p.tile_counters + pc.tile) : "memory");
-                        s_last = (prev == pc.n_pieces - 1);
-                        if (s_last) p.tile_counters[pc.tile] = 0;
+                        if (cp.test_stuck && oi == 0 && pc.index != 0) {
+                            s_last = 0;             // test hook: this part is never announced, the tile never finishes
+                        } else {
+                            int prev;
+                            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                                         : "=r"(prev) : "l"(p.tile_counters + pc.tile) : "memory");
+                            s_last = (prev == pc.n_pieces - 1);
+                            if (s_last) p.tile_counters[pc.tile] = 0;
+                        }
                     }
                     epi_bar();
                     if (et == 0) PASS_TRACE(oi, 5);

@@ -141,7 +141,14 @@ struct pass_ctx {
     bool attn_long = false;       // this step's contexts are long: twice as many attention slices (see step_launch)
     int attn_long_from = 3072;    // PASS_ATTN_LONG_FROM: cached positions from which a step counts as long
     bool attn_cluster = true;     // PASS_ATTN_NO_CLUSTER: merge attention slices through global memory
-    int attn_debug_stale = 0;     // PASS_ATTN_STALE=n: attention's early part works from a cache length n short
+    int attn_debug_stale = 0;     // pass_debug_set(PASS_HOOK_ATTN_STALE, n): attention's early part works from a cache length n short
+    int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
+    // Function attributes and occupancy answers belong to the device the context lives on, so they are
+    // remembered per context, never per process.
+    size_t gemm_smem_set = 0;
+    std::map<int, bool> attn_attr_set;         // by kernel instance
+    std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
+    cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
     bool use_tc = false;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
     int trace_launch = 0;
@@ -196,6 +203,24 @@ struct pass_ctx {
     do {                                                              \
         kern<<<(grid), (block), 0, (ctx)->stream>>>(__VA_ARGS__);     \
         (ctx)->launches++;                                            \
+    } while (0)
+
+// Launches and attribute calls made deep inside the enqueue helpers report here; the entry points
+// turn the first recorded failure into PASS_ERR_CUDA (launch_failed) before they hand anything back.
+static void note_err(pass_ctx* c, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return;
+    if (c->launch_err == cudaSuccess) c->launch_err = e;
+    if (getenv("PASS_LOG")) fprintf(stderr, "[pass] %s failed: %s\n", what, cudaGetErrorString(e));
+}
+static bool launch_failed(pass_ctx* c) {
+    const cudaError_t e = c->launch_err;
+    c->launch_err = cudaSuccess;
+    return e != cudaSuccess;
+}
+#define CHECK_LAUNCHES(ctx)                                   \
+    do {                                                      \
+        if (launch_failed(ctx)) return PASS_ERR_CUDA;         \
+        CUDA_TRY(cudaGetLastError());                         \
     } while (0)
 
 // ------------------------------------------------------------------------------- small kernels
@@ -317,7 +342,7 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     cp.n_ops = n_ops;
     cp.stages = ops[0].p.stages;
     cp.npad = ops[0].p.npad;
-    cp.test_stuck = getenv("PASS_GEMM_TEST_STUCK") ? 1 : 0;
+    cp.test_stuck = c->gemm_test_stuck;
     cp.hold = getenv("PASS_GEMM_HOLD") ? atoi(getenv("PASS_GEMM_HOLD")) : 0;
     cp.op_done = c->d_chain_flags;
     for (int j = 0; j < kMaxOps; j++) {
@@ -342,13 +367,12 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     for (int j = n_ops; j < kMaxOps; j++)
         for (int q = 0; q < 4; q++) maps.m[j][q] = ops[0].a0;
     const size_t smem = (size_t)cp.stages * (kATileBytes + cp.npad * 128) + 1024;
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-        cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem > c->gemm_smem_set) {
+        note_err(c, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "k_gemm_tc shared memory size");
         // all of the SM's L1/shared storage as shared memory: lets the CTA of the next launch become
         // resident (and start pulling weights) while this launch's CTA is still running
-        cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        smem_set = smem;
+        note_err(c, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_gemm_tc carveout");
+        c->gemm_smem_set = smem;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -364,14 +388,14 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = c->use_pdl ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, cp);
+    note_err(c, cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, cp), "k_gemm_tc launch");
     c->launches++;
 }
 
 // Start of a forward: the chain's completion counters go back to zero (on the device, in stream order, and
 // in the host's mirror).  Also what makes the next forward right after one that was abandoned on a time-out.
 static void chain_counters_clear(pass_ctx* c) {
-    cudaMemsetAsync(c->d_chain_flags, 0, sizeof(int) * kMaxOps, c->stream);
+    note_err(c, cudaMemsetAsync(c->d_chain_flags, 0, sizeof(int) * kMaxOps, c->stream), "chain counter clear");
     for (int j = 0; j < kMaxOps; j++) c->chain_done_total[j] = 0;
 }
 
@@ -387,10 +411,10 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
 template <int DH, int MT, bool CL>
 static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
-    static bool set = false;
+    bool& set = c->attn_attr_set[DH * 8 + MT * 2 + (CL ? 1 : 0)];
     if (!set) {
-        cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_attn_fd carveout");
         set = true;
     }
     cudaLaunchConfig_t cfg;
@@ -413,19 +437,21 @@ static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     }
     cfg.attrs = at;
     cfg.numAttrs = na;
-    cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL>, ap);
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL>, ap), "k_attn_fd launch");
     c->launches++;
 }
 
 // Can the slices of every (sequence, head) run as one cluster each, all at the same time?  Asked once per
-// kernel instance and slice count; if not (or with more than 8 slices) the merge goes through global memory.
+// context, kernel instance, slice count and batch; if not (or with more than 8 slices) the merge goes through
+// global memory.
 template <int DH, int MT>
 static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
     if (!c->attn_cluster || n_split < 2 || n_split > 8) return false;
-    static int cached_split = -1, cached_max = 0;
-    if (cached_split != n_split) {
+    const int key = ((DH * 8 + MT) * 32 + n_split) * 256 + n_seq;
+    auto it = c->attn_cluster_max.find(key);
+    if (it == c->attn_cluster_max.end()) {
         constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
-        cudaFuncSetAttribute(k_attn_fd<DH, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
         cfg.gridDim = dim3(c->md.H, n_seq, n_split);
@@ -438,10 +464,9 @@ static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
         cfg.numAttrs = 1;
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
-        cached_split = n_split;
-        cached_max = n;
+        it = c->attn_cluster_max.emplace(key, n).first;
     }
-    return cached_max >= c->md.H * n_seq;
+    return it->second >= c->md.H * n_seq;
 }
 
 template <int DH, int MT>
@@ -634,7 +659,7 @@ static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool w
         }
     }
     c->last_rows = n;
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     return PASS_OK;
 }
 
@@ -720,7 +745,6 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         c->attn_cluster = getenv("PASS_ATTN_NO_CLUSTER") == nullptr;
         if (const char* e = getenv("PASS_ATTN_LONG_FROM")) c->attn_long_from = std::max(0, atoi(e));
-        if (const char* e = getenv("PASS_ATTN_STALE")) c->attn_debug_stale = std::max(0, atoi(e));
         c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) == cudaSuccess &&
@@ -799,7 +823,7 @@ int pass_load_weights(pass_ctx* c, const pass_weights* w) {
 int pass_reset(pass_ctx* c, int seq) {
     if (!c || seq < 0 || seq >= c->md.B) return PASS_ERR_INVALID_ARG;
     LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, 0, 0, 0, 1);
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->len_ub[seq] = 0;
     c->prefilled[seq] = 0;
@@ -816,7 +840,7 @@ int pass_set_state(pass_ctx* c, int seq, int len, int32_t pending) {
     if (!c || seq < 0 || seq >= c->md.B || len < 0 || pending < 0 || pending >= c->md.V) return PASS_ERR_INVALID_ARG;
     if (len > c->md.cap) return PASS_ERR_CAPACITY;
     LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 1, len, 0, 1, (int)pending, 0);
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->len_ub[seq] = len;
     c->prefilled[seq] = 1;
@@ -841,7 +865,7 @@ int pass_forward_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, floa
         CUDA_TRY(cudaMemcpyAsync(logits_out_device, c->d_logits, sizeof(float) * (size_t)n * c->md.V,
                                  cudaMemcpyDeviceToDevice, c->stream));
     LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, commit, 0, 0, 0);
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->len_ub[seq] += commit;
     return PASS_OK;
@@ -867,11 +891,21 @@ int pass_prefill(pass_ctx* c, int seq, const int32_t* tokens, int n) {
         CUDA_TRY(cudaStreamSynchronize(c->stream));   // pin_tok is reused by the next chunk
     }
     LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, 0, 1, (int)tokens[n - 1], 0);
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     c->len_ub[seq] = n - 1;
     c->prefilled[seq] = 1;
     return PASS_OK;
+}
+
+// A launch that gave up on a bounded wait may leave its cross-CTA scratch half used: hand-over words
+// that are not EMPTY, arrival counters of split tiles and of attention slices that are not zero.  All of
+// it goes back to the idle state, in stream order, before the next launch.
+static cudaError_t scrub_after_timeout(pass_ctx* c) {
+    cudaError_t e = cudaMemsetAsync(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps, c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->d_counters, 0, 4096 * sizeof(int), c->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_cnt, 0, (size_t)c->md.B * c->md.H * sizeof(int), c->stream);
+    return e;
 }
 
 static int step_checks(pass_ctx* c, int k, float T, const void* uniforms) {
@@ -917,7 +951,10 @@ static int step_launch(pass_ctx* c, int k, float T) {
             CUDA_TRY(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
             enqueue_step_any(c, k);
             cudaError_t e = cudaStreamEndCapture(c->stream, &g);
-            if (e != cudaSuccess || !g) return PASS_ERR_CUDA;
+            if (e != cudaSuccess || !g || launch_failed(c)) {
+                if (g) cudaGraphDestroy(g);
+                return PASS_ERR_CUDA;
+            }
             cudaGraphExec_t ge = nullptr;
             e = cudaGraphInstantiate(&ge, g, 0);
             cudaGraphDestroy(g);
@@ -930,7 +967,7 @@ static int step_launch(pass_ctx* c, int k, float T) {
         c->last_step_launches = c->graph_launches[gkey];
     } else {
         enqueue_step_any(c, k);
-        CUDA_TRY(cudaGetLastError());
+        CHECK_LAUNCHES(c);
         c->last_step_launches = c->launches;
     }
     c->last_rows = c->md.B * (1 + 2 * k);
@@ -960,8 +997,7 @@ int pass_step_collect(pass_ctx* c, int32_t* out_tokens, int32_t* n_out) {
     const int status = *c->pin_status;
     if (status != 0) {
         CUDA_TRY(cudaMemsetAsync(c->d_status, 0, sizeof(int), c->stream));
-        if ((status & kStatusTimeout) && c->d_ll)       // an abandoned launch may have left words in the slots
-            CUDA_TRY(cudaMemsetAsync(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps, c->stream));
+        if ((status & kStatusTimeout) && c->d_ll) CUDA_TRY(scrub_after_timeout(c));
         CUDA_TRY(cudaStreamSynchronize(c->stream));
         if (status & kStatusTimeout) return PASS_ERR_TIMEOUT;
         if (status & kStatusNonFinite) return PASS_ERR_NONFINITE;
@@ -1066,7 +1102,7 @@ static int kv_copy(pass_ctx* c, int seq, int layer, int pos0, int n, void* k, vo
             if (gather) CUDA_TRY(cudaMemcpyAsync(hp, stage, cn * rowb, cudaMemcpyDeviceToHost, c->stream));
             CUDA_TRY(cudaStreamSynchronize(c->stream));
         }
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     return PASS_OK;
 }
 
@@ -1156,7 +1192,10 @@ static int debug_status(pass_ctx* c) {
     CUDA_TRY(cudaMemcpy(&status, c->d_status, 4, cudaMemcpyDeviceToHost));
     if (status) {
         CUDA_TRY(cudaMemset(c->d_status, 0, 4));
-        if ((status & kStatusTimeout) && c->d_ll) CUDA_TRY(cudaMemset(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps));
+        if ((status & kStatusTimeout) && c->d_ll) {
+            CUDA_TRY(scrub_after_timeout(c));
+            CUDA_TRY(cudaStreamSynchronize(c->stream));
+        }
         return (status & kStatusTimeout) ? PASS_ERR_TIMEOUT : PASS_ERR_STATE;
     }
     return PASS_OK;
@@ -1174,7 +1213,7 @@ int pass_debug_linear(pass_ctx* c, int which, int layer, const float* x_device, 
     LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x_device, K, which == 6 ? c->d_act_bf : c->d_xn_bf, npad_for(R) / 2);
     const int rc = enqueue_debug_linear(c, which, layer, R, y_device);
     if (rc != PASS_OK) return rc;
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     return debug_status(c);
 }
@@ -1214,7 +1253,7 @@ int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float*
     CUDA_TRY(cudaEventRecord(e0, c->stream));
     for (int i = 0; i < n_launches; i++) one(i);
     CUDA_TRY(cudaEventRecord(e1, c->stream));
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     CUDA_TRY(cudaEventElapsedTime(ms_total, e0, e1));
     cudaEventDestroy(e0);
@@ -1223,12 +1262,20 @@ int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float*
 }
 
 // ------------------------------------------------------------------------------- no-allocation linear
-// Scratch of the split-K GEMM (partial sums of tiles shared by several CTAs + one counter per tile)
-// kept inside the library image instead of in caller-provided memory.  Sized for at most
-// kStaticMaxRows token rows; every GPU that loads the library carries these bytes until exit.
+// Scratch of the split-K GEMM (the words through which CTAs that share an output tile hand their
+// partial sums to the one that finishes it) kept inside the library image instead of in
+// caller-provided memory.  Sized for at most kStaticMaxRows token rows; every GPU that loads the
+// library carries these bytes until exit.
+//
+// Only ONE hand-over protocol ever touches the array: EMPTY-or-value words.  The GEMM kernel picks
+// that protocol when the token rows are padded to 16 per half (rh == 16) and arrival counters with
+// float4 partial slots otherwise, so this entry point pads EVERY call to 16 rows, also calls of 1 to
+// 8 rows that the step itself would run with 8 rows per half.  A counter-protocol launch would leave
+// its partial sums in the words, and a later finisher that polls a word before its contributor's
+// store has landed would take such a leftover for the value.
 constexpr int kStaticMaxRows = 16;
 constexpr size_t kStaticPartialBytes = (size_t)kMaxCtas * 2 * kStaticMaxRows * kTileN * sizeof(float);
-constexpr size_t kStaticCounterBytes = 4096 * sizeof(int);
+constexpr size_t kStaticCounterBytes = 4096 * sizeof(int);      // not used any more; keeps the array's size
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartialBytes + kStaticCounterBytes];
 
 // Device address of g_static_scratch per device ordinal.  In host code the symbol's name is only a
@@ -1254,15 +1301,14 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     if (!g_static_scratch_addr[dev]) {          // first call on this device
         void* ptr = nullptr;
         CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
-        // the hand-over slots start out EMPTY (all bits set); every call leaves them that way
+        // the hand-over words start out EMPTY (all bits set); every call leaves them that way
         CUDA_TRY(cudaMemsetAsync(ptr, 0xFF, kStaticPartialBytes, c->stream));
         g_static_scratch_addr[dev] = ptr;
     }
     char* scratch = (char*)g_static_scratch_addr[dev];
-    // the tile counters must start at zero; the partial sums are always written before they are read
-    CUDA_TRY(cudaMemsetAsync(scratch + kStaticPartialBytes, 0, kStaticCounterBytes, c->stream));
 
-    const int d = c->md.d, f = c->md.f, npad = npad_for(R);
+    const int d = c->md.d, f = c->md.f;
+    const int npad = 2 * kStaticMaxRows;        // always 16 rows per half: the EMPTY-or-value protocol (see above)
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     const int K = which == 6 ? f : d;
@@ -1282,20 +1328,38 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
         default: a0 = &c->tm_wg[layer]; a1 = &c->tm_wu[layer]; N = ((f + 63) / 64) * 128; break;
     }
     const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
-    if (n_tiles > (int)(kStaticCounterBytes / sizeof(int))) return PASS_ERR_CAPACITY;
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
     p.logits = y_device;
-    p.partial_ws = (float*)scratch;          // never used with <= 16 rows
+    p.partial_ws = nullptr;                  // the counter protocol is never taken with rh == 16
+    p.tile_counters = nullptr;
     p.ll_ws = (float*)scratch;
-    p.tile_counters = (int*)(scratch + kStaticPartialBytes);
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
-    CUDA_TRY(cudaGetLastError());
+    CHECK_LAUNCHES(c);
     CUDA_TRY(cudaStreamSynchronize(c->stream));
     const int rc = debug_status(c);
     if (rc == PASS_ERR_TIMEOUT)     // an abandoned launch may have left words in the shared slots
         CUDA_TRY(cudaMemset(scratch, 0xFF, kStaticPartialBytes));
     return rc;
+}
+
+int pass_debug_set(pass_ctx* c, int hook, int value) {
+    if (!c || value < 0) return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    switch (hook) {
+        case PASS_HOOK_GEMM_STUCK: c->gemm_test_stuck = value ? 1 : 0; break;
+        case PASS_HOOK_ATTN_STALE: c->attn_debug_stale = value; break;
+        default: return PASS_ERR_INVALID_ARG;
+    }
+    // the hooks are part of the launch parameters, which captured graphs hold by value
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+    c->graphs.clear();
+    c->graph_launches.clear();
+    return PASS_OK;
 }
 
 int pass_debug_schedule(int n_tiles, int kb_per_tile, int n_ctas, int cta, int it, int32_t* out) {

@@ -141,9 +141,10 @@ def test_changing_k_and_temperature_between_steps(tiny_w):
 
 
 def test_bf16_changing_k_alternates_between_the_two_partial_sum_protocols():
-    """k = 4, 1, 0 (up to 16 rows: partial sums handed over through EMPTY-or-value words, with 9, 3 and 1
-    live rows) and k = 8 (17 rows: arrival counters) in one context, back and forth: each protocol must
-    find its scratch as it left it, and the graphs of the different k must not disturb each other."""
+    """k = 4 (9 rows, padded to 16 per half: partial sums handed over through EMPTY-or-value words) and
+    k = 0, 1, 2 (1, 3, 5 rows) or k = 8 (17 rows), which use arrival counters, in one context, back and
+    forth: each protocol must find its scratch as it left it, and the graphs of the different k must not
+    disturb each other."""
     from parity_util import lockstep, make_pair
     prompt = si.make_prompt(TINY_BF16, 40)
     ctx, oracles, _ = make_pair(TINY_BF16, 1, 400, [prompt], seed=1)
@@ -258,14 +259,13 @@ def test_unk_lookahead_baseline_runs_through_the_same_path():
 
 
 # ------------------------------------------------------------------ a wait that runs out
-def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(monkeypatch):
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     """Every device-side wait has a limit.  The hook makes the contributors of the first GEMM of each
     launch keep their partial sums to themselves, so the CTAs that finish those tiles wait for words that
     never come: after the limit (0.2 s) they give up, the other roles follow, the step reports TIMEOUT,
     the sequence state is untouched, and the next steps are correct again."""
     import paper_2311_13581_b200 as pb
     from parity_util import lockstep
-    monkeypatch.setenv("PASS_NO_GRAPH", "1")          # the hook is read when a launch is built
     shape = SEVENB_2L
     w = si.make_weights(shape, seed=0, device="cuda:0")
     w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
@@ -279,13 +279,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(monkeypat
     orc.Q_dft, orc.k_prev, orc.T_prev, orc.last_logits = np.zeros((0, shape.vocab)), None, None, None
     stats, _ = lockstep(ctx, [orc], 4, 0.0, 2)
     len_before = ctx.get_debug(pb.PASS_DBG_KV_LEN).copy()
-    monkeypatch.setenv("PASS_GEMM_TEST_STUCK", "1")
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 1)
     with pytest.raises(pb.PassError) as e:
         ctx.step(4, 0.0, None)
     assert "timed out" in str(e.value)
-    monkeypatch.delenv("PASS_GEMM_TEST_STUCK")
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 0)
     assert (ctx.get_debug(pb.PASS_DBG_KV_LEN) == len_before).all()
     stats, _ = lockstep(ctx, [orc], 4, 0.0, 2, step0=2)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    # the same with a step that uses arrival counters (k = 1: 3 rows): an abandoned launch leaves
+    # counters half counted, and the steps after it must find them at zero again
+    stats, _ = lockstep(ctx, [orc], 1, 0.0, 2, step0=4)
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 1)
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(1, 0.0, None)
+    assert "timed out" in str(e.value)
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 0)
+    stats, _ = lockstep(ctx, [orc], 1, 0.0, 3, step0=6)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    stats, _ = lockstep(ctx, [orc], 4, 0.0, 2, step0=9)
     assert stats["max_logit_err"] <= 1e-2, stats
     ctx.close()
 
@@ -377,15 +389,15 @@ def test_tiny_bf16_long_prompt_many_key_blocks(k):
     ctx.close()
 
 
-def test_attention_restarts_when_its_early_fetch_used_outdated_row_tables(monkeypatch):
+def test_attention_restarts_when_its_early_fetch_used_outdated_row_tables():
     """The attention kernel fetches old cache rows before its queries exist, from row tables it reads
     ahead of the kernel it depends on, and starts over if those turn out to be outdated.  On a normal
     run they never are, so the hook makes the early part work from a cache length 70 short (another
     split of the keys, other blocks in the ring): results must not change."""
     from parity_util import lockstep, make_pair
-    monkeypatch.setenv("PASS_ATTN_STALE", "70")
     prompt = si.make_prompt(TINY_BF16, 333)
     ctx, oracles, _ = make_pair(TINY_BF16, 1, 333 + 80, [prompt], seed=1)
+    ctx.debug_set(_pb().PASS_HOOK_ATTN_STALE, 70)
     stats, _ = lockstep(ctx, oracles, 4, 0.8, 4, check_A=False)
     assert stats["max_logit_err"] <= 1e-2, stats
     stats, _ = lockstep(ctx, oracles, 4, 0.0, 3, step0=4, check_A=True)

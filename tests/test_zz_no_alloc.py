@@ -42,6 +42,30 @@ def test_noalloc_linear_matches_ordinary_entry_twice_in_a_row():
     ctx.close()
 
 
+def test_noalloc_linear_alternating_row_counts_never_sees_leftovers():
+    """Calls of 1 to 8 rows and of 9 to 16 rows, back and forth, many times, on matrices whose output
+    tiles are each shared by several CTAs (K = 1384 and 512 against 148 CTAs).  In the step these two
+    row ranges hand their partial sums over in different ways; the built-in array must only ever see the
+    empty-or-value words, whatever the row count, or a later call could pick up an earlier call's
+    partial sums.  Every result is compared bit for bit with the ordinary entry point."""
+    import paper_2311_13581_b200 as pb
+    w = si.make_weights(MID, seed=4)
+    ctx = pb.PassContext(MID, si.weights_to(w, "cuda:0"), 1, 64)
+    g = torch.Generator().manual_seed(12)
+    calls = 0
+    for rep in range(12):
+        for which, layer, R in ((6, 1, 5), (6, 1, 12), (3, 0, 8), (3, 0, 9), (6, 0, 1), (6, 0, 16), (8, 1, 3), (7, 0, 13)):
+            K = MID.d_ffn if which == 6 else MID.d_model
+            x = torch.randn(R, K, generator=g).cuda()
+            ref = ctx.debug_linear(which, layer, x)
+            y = torch.empty_like(ref)
+            got = ctx.linear_noalloc(which, layer, x, y)
+            assert torch.equal(got, ref), (rep, which, layer, R)
+            calls += 1
+    assert calls == 96
+    ctx.close()
+
+
 def test_noalloc_linear_rejects_more_rows_than_its_scratch_holds():
     import paper_2311_13581_b200 as pb
     w = si.make_weights(MID, seed=4)
