@@ -52,6 +52,8 @@ struct GemmParams {
     int n_tiles, kb_per_tile;
     int seg_tiles0, seg_tiles1;    // plain mode: tiles of weight map 0 and 1 (the rest is map 2)
     int interleave;                // 1: tile t = rows [64t, 64t+64) of map 0 (gate) and of map 1 (up)
+    int packed;                    // 1: the weight maps are over the packed copy [tile][k-block][box rows][64]
+                                   // (see k_pack_weight): a box is addressed by its number, not by row and column
     int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
     int stages;
     int epi;
@@ -491,7 +493,9 @@ struct ChainParams {
     unsigned long long* trace;     // optional %globaltimer stamps [kMaxOps][CTA][8] of this launch (nullptr = off)
     GemmParams op[kMaxOps];
 };
-#define PASS_TRACE(oi, slot) do { if (cp.trace) cp.trace[((size_t)(oi) * gridDim.x + blockIdx.x) * 8 + (slot)] = global_ns(); } while (0)
+// Only every 16th CTA leaves stamps: reads of %globaltimer from all CTAs at once queue up behind one another
+// (tens of microseconds for 148 readers) and would stretch the very hand-overs the trace is meant to show.
+#define PASS_TRACE(oi, slot) do { if (cp.trace && (blockIdx.x & 15) == 0) cp.trace[((size_t)(oi) * gridDim.x + blockIdx.x) * 8 + (slot)] = global_ns(); } while (0)
 
 __device__ __forceinline__ bool wait_count(const int* counter, int target, volatile int* s_abort, int* g_status) {
     const long long t0 = clock64();
@@ -509,7 +513,9 @@ __device__ __forceinline__ bool wait_count(const int* counter, int target, volat
     }
 }
 
-// weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box
+// weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box.
+// The coordinates of k-block kb are (kb * kBlockK, y) in a row-major matrix and (0, y * kb_per_tile +
+// kb * box rows) in the packed copy; weight_xy turns the one into the other.
 __device__ __forceinline__ void weight_box(const GemmParams& p, const CUtensorMap* m4, int tile, int box,
                                            const CUtensorMap*& m, int& y) {
     if (p.interleave) {
@@ -524,6 +530,15 @@ __device__ __forceinline__ void weight_box(const GemmParams& p, const CUtensorMa
             if (tl >= p.seg_tiles1) { tl -= p.seg_tiles1; m = m4 + 2; }
         }
         y = tl * kTileN;
+    }
+}
+__device__ __forceinline__ void weight_xy(const GemmParams& p, int y_rowmajor, int kb, int& x, int& y) {
+    if (p.packed) {
+        x = 0;
+        y = y_rowmajor * p.kb_per_tile + kb * (p.interleave ? 64 : kTileN);
+    } else {
+        x = kb * kBlockK;
+        y = y_rowmajor;
     }
 }
 
@@ -622,7 +637,9 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         const uint32_t parity = ((fill / S) & 1) ^ 1;
                         if (!mbar_wait(bar_empty + 8 * s, parity, &s_abort, cp.status)) { ok = false; break; }
                         mbar_expect_tx(bar_full + 8 * s, a_box_bytes);
-                        tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
+                        int wx, wy;
+                        weight_xy(p, y, kb, wx, wy);
+                        tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, wx, wy, pol_w);
                         fill++;
                         *(volatile int*)&s_issued = fill;
                     }
@@ -656,7 +673,9 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         const uint32_t dst = tiles_base + s * stage_bytes;
                         if (p.interleave) {
                             mbar_expect_tx(bar_full + 8 * s, stage_bytes - a_box_bytes);
-                            tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, kb * kBlockK, y, pol_w);
+                            int wx, wy;
+                            weight_xy(p, y, kb, wx, wy);
+                            tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, wx, wy, pol_w);
                         } else {
                             mbar_expect_tx(bar_full + 8 * s, stage_bytes - kATileBytes);
                         }

@@ -354,6 +354,26 @@ __global__ void k_split_rows(const float* __restrict__ x, int K, __nv_bfloat16* 
     out[(size_t)(lo_row0 + r) * K + c] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// Weight matrix W[N][K] (row-major bf16) copied into the order the streaming GEMM reads it:
+// [tile][k-block][box_rows][64] - every (tile, k-block) box is one contiguous run of box_rows * 128
+// bytes instead of box_rows pieces of 128 bytes that lie a whole matrix row apart.  Rows and columns
+// beyond the matrix are zeros.  One thread moves 16 bytes.
+__global__ void k_pack_weight(const __nv_bfloat16* __restrict__ W, int N, int K, int box_rows, int n_tiles,
+                              int kb_per_tile, __nv_bfloat16* __restrict__ out) {
+    const size_t total = (size_t)n_tiles * kb_per_tile * box_rows * 8;      // 16-byte chunks
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c8 = (int)(i & 7);
+        const size_t rest = i >> 3;
+        const int r = (int)(rest % box_rows);
+        const size_t box = rest / box_rows;
+        const int kb = (int)(box % kb_per_tile), tile = (int)(box / kb_per_tile);
+        const int row = tile * box_rows + r, col = kb * 64 + c8 * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row < N && col < K) v = *reinterpret_cast<const uint4*>(W + (size_t)row * K + col);   // K is a multiple of 8
+        reinterpret_cast<uint4*>(out)[i] = v;
+    }
+}
+
 // F[r][j] = silu(G[r][j]) * U[r][j], GU: [R][2f] (gate | up)
 __global__ void k_swiglu(const float* __restrict__ gu, int f, float* __restrict__ act) {
     const int r = blockIdx.y;

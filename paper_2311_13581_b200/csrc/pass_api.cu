@@ -36,8 +36,14 @@ struct Layout {
     size_t xn_bf, attn_bf, act_bf, q_out, sumsq_a, sumsq_b, partial_ws, counters;   // tensor-core path
     size_t ll_ws;
     size_t attn_po, attn_pml, attn_cnt, chain_flags;
+    size_t packed, packed_bytes;       // the weights in streaming order (see k_pack_weight)
     size_t total;
 };
+
+// Bytes of one weight matrix [N][K] in the packed order: whole boxes of box_rows x 64 elements.
+size_t packed_matrix_bytes(size_t N, size_t K, size_t box_rows) {
+    return ((N + box_rows - 1) / box_rows) * ((K + 63) / 64) * box_rows * 128;
+}
 
 bool config_ok(const pass_config* c) {
     if (!c) return false;
@@ -88,6 +94,7 @@ Layout make_layout(const pass_config& c) {
     L.scratch = cv.take(B * kChunks * 8);
     L.xn_bf = L.attn_bf = L.act_bf = L.q_out = L.sumsq_a = L.sumsq_b = L.partial_ws = L.counters = 0;
     L.attn_po = L.attn_pml = L.attn_cnt = L.chain_flags = 0;
+    L.packed = L.packed_bytes = 0;
     if (c.dtype == PASS_DTYPE_BF16) {
         L.xn_bf = cv.take(2 * R * d * 2);
         L.attn_bf = cv.take(2 * R * d * 2);
@@ -103,6 +110,9 @@ Layout make_layout(const pass_config& c) {
         L.attn_pml = cv.take(slices * 32 * 2 * 4);
         L.attn_cnt = cv.take(B * c.n_heads * 4);
         L.chain_flags = cv.take(2 * kMaxOps * 4);
+        L.packed_bytes = (size_t)c.n_layers * (4 * packed_matrix_bytes(d, d, 128) + 2 * packed_matrix_bytes(f, d, 64) +
+                                               packed_matrix_bytes(d, f, 128)) + packed_matrix_bytes(V, d, 128);
+        L.packed = cv.take(L.packed_bytes);
     }
     L.total = cv.off;
     return L;
@@ -150,6 +160,8 @@ struct pass_ctx {
     std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
     bool use_tc = false;
+    bool packed = false;               // the GEMMs stream the packed copy of the weights (PASS_NO_PACK: the caller's matrices)
+    char* d_packed = nullptr;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
     int trace_launch = 0;
     int chain_done_total[kMaxOps] = {0, 0, 0, 0};   // host mirror of what the counters reach (see launch_chain)
@@ -281,6 +293,19 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t c
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The packed copy of a matrix as a tensor map: n_boxes boxes of box_rows x 64 elements, one after another.
+static bool make_map_packed(CUtensorMap* m, const void* base, uint64_t n_boxes, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kBlockK, n_boxes * box_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kBlockK * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 static int npad_for(int R) { return ((2 * R + 15) / 16) * 16; }
 
 static int gemm_stages(int npad) {
@@ -323,6 +348,7 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     p.eps = c->md.eps;
     p.md = c->md;
     p.xn_lo_row0 = npad / 2;
+    p.packed = c->packed ? 1 : 0;
     return p;
 }
 
@@ -331,6 +357,15 @@ struct ChainOp {
     GemmParams p;
     CUtensorMap a0, a1, a2, b;
 };
+
+// The tail of the verify scratch (E, [kMaxRows][V] doubles) doubles as the trace buffer: its rows beyond the
+// first half are only used by steps of more than 64 rows.  nullptr when E is too small for that.
+constexpr int kTraceLaunches = 48;
+static unsigned long long* trace_base(pass_ctx* c) {
+    const size_t total = (size_t)kMaxRows * c->md.V, need = (size_t)kTraceLaunches * kMaxOps * kMaxCtas * 8;
+    if (need > total / 2) return nullptr;
+    return (unsigned long long*)c->vb.E + (total - need);
+}
 
 // Launch up to kMaxOps dependent GEMMs as ONE kernel (see k_gemm_tc).  GEMM j of the chain gets its own
 // partial-sum region and tile counters, because its split tiles may be in flight while GEMM j-1 is
@@ -352,8 +387,8 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
         cp.op_target[j] = c->chain_done_total[j];
     }
     cp.status = c->d_status;
-    if (c->trace && c->trace_launch < 48)      // the verify scratch (E) doubles as the trace buffer
-        cp.trace = (unsigned long long*)c->vb.E + (size_t)(c->trace_launch++) * kMaxOps * kMaxCtas * 8;
+    if (c->trace && c->trace_launch < kTraceLaunches && trace_base(c))
+        cp.trace = trace_base(c) + (size_t)(c->trace_launch++) * kMaxOps * kMaxCtas * 8;
     const size_t region = (size_t)kMaxCtas * 2 * kMaxRows * kTileN;      // floats per GEMM of the chain
     for (int j = 0; j < n_ops; j++) {
         if (ops[j].p.partial_ws == c->d_partial) {
@@ -741,6 +776,8 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_attn_pml = (float*)(w + L.attn_pml);
         c->d_attn_cnt = (int*)(w + L.attn_cnt);
         c->d_chain_flags = (int*)(w + L.chain_flags);
+        c->d_packed = w + L.packed;
+        c->packed = getenv("PASS_NO_PACK") == nullptr;
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         c->attn_cluster = getenv("PASS_ATTN_NO_CLUSTER") == nullptr;
@@ -765,7 +802,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     // zero the small state region; rotary frequencies theta^(-2i/d_head) in float64
     if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     if (cfg->dtype == PASS_DTYPE_BF16 &&
-        cudaMemsetAsync(w + L.xn_bf, 0, L.total - L.xn_bf, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+        cudaMemsetAsync(w + L.xn_bf, 0, L.packed - L.xn_bf, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     // the hand-over slots of the <=16-row GEMMs are EMPTY (all bits set) whenever no launch is using them
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.ll_ws, 0xFF, kLLRegionBytes * kMaxOps, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
@@ -803,12 +840,28 @@ int pass_load_weights(pass_ctx* c, const pass_weights* w) {
         std::vector<CUtensorMap>* tms[] = {&c->tm_wq, &c->tm_wk, &c->tm_wv, &c->tm_wo, &c->tm_wg, &c->tm_wu, &c->tm_wd};
         const std::vector<const void*>* ws[] = {&c->wq, &c->wk, &c->wv, &c->wo, &c->wg, &c->wu, &c->wd};
         const int rows[] = {d, d, d, d, f, f, d}, cols[] = {d, d, d, d, d, d, f};
+        // With packing on, every matrix is first copied into streaming order inside the workspace and
+        // the map is laid over the copy; the caller's matrices stay as they are.
+        char* pk = c->d_packed;
+        auto weight_map = [&](CUtensorMap* m, const void* W, int N, int K, int box_rows) -> bool {
+            if (!c->packed) return make_map(m, W, N, K, box_rows);
+            const int n_tiles = (N + box_rows - 1) / box_rows, kbpt = (K + kBlockK - 1) / kBlockK;
+            const size_t bytes = packed_matrix_bytes(N, K, box_rows);
+            if (pk + bytes > c->d_packed + c->L.packed_bytes) return false;
+            const int blocks = (int)std::min<size_t>(148 * 16, (bytes / 16 + 255) / 256);
+            LAUNCH(c, k_pack_weight, blocks, 256, (const __nv_bfloat16*)W, N, K, box_rows, n_tiles, kbpt, (__nv_bfloat16*)pk);
+            const bool ok = make_map_packed(m, pk, (uint64_t)n_tiles * kbpt, box_rows);
+            pk += bytes;
+            return ok;
+        };
         for (int i = 0; i < 7; i++) {
             tms[i]->resize(nl);
             for (int l = 0; l < nl; l++)
-                if (!make_map(&(*tms[i])[l], (*ws[i])[l], rows[i], cols[i], (i == 4 || i == 5) ? 64 : 128)) return PASS_ERR_CUDA;
+                if (!weight_map(&(*tms[i])[l], (*ws[i])[l], rows[i], cols[i], (i == 4 || i == 5) ? 64 : 128)) return PASS_ERR_CUDA;
         }
-        if (!make_map(&c->tm_lm, c->lm_head, c->md.V, d, 128)) return PASS_ERR_CUDA;
+        if (!weight_map(&c->tm_lm, c->lm_head, c->md.V, d, 128)) return PASS_ERR_CUDA;
+        CHECK_LAUNCHES(c);
+        CUDA_TRY(cudaStreamSynchronize(c->stream));
         c->tm_wg_plain.resize(nl);
         c->tm_wu_plain.resize(nl);
         for (int l = 0; l < nl; l++) {
@@ -1125,8 +1178,9 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         return PASS_OK;
     }
     if (what == PASS_DBG_TRACE) {
-        const size_t n = std::min(bytes, (size_t)48 * kMaxOps * kMaxCtas * 8 * 8);
-        CUDA_TRY(cudaMemcpy(dst, c->vb.E, n, cudaMemcpyDeviceToHost));
+        if (!trace_base(c)) return PASS_ERR_STATE;
+        const size_t n = std::min(bytes, (size_t)kTraceLaunches * kMaxOps * kMaxCtas * 8 * 8);
+        CUDA_TRY(cudaMemcpy(dst, trace_base(c), n, cudaMemcpyDeviceToHost));
         c->trace_launch = 0;
         return PASS_OK;
     }
@@ -1182,6 +1236,7 @@ static int enqueue_debug_linear(pass_ctx* c, int which, int layer, int R, float*
     const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
+    if (which == 4 || which == 5) p.packed = 0;     // gate or up alone: 128-row boxes over the caller's matrix
     p.logits = y_device;
     launch_gemm(c, *a0, a1 ? *a1 : *a0, *a0, which == 6 ? bm->act : bm->xn, p);
     return PASS_OK;
@@ -1330,6 +1385,7 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     const int n_tiles = which == 8 ? (f + 63) / 64 : (N + kTileN - 1) / kTileN;
     GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
     p.interleave = which == 8;
+    if (which == 4 || which == 5) p.packed = 0;
     p.logits = y_device;
     p.partial_ws = nullptr;                  // the counter protocol is never taken with rh == 16
     p.tile_counters = nullptr;

@@ -110,6 +110,23 @@ _S_PROMPT, _S_UNIF = 1 << 20, 1 << 21
 _TORCH_DTYPE = {"fp32": torch.float32, "bf16": torch.bfloat16}
 
 
+_LAYER_NAMES = ["wq", "wk", "wv", "wo", "wg", "wu", "wd"]
+
+
+def make_layer_weights(shape: ModelShape, layer: int, seed: int = 0, device="cpu", std: float = 0.02
+                       ) -> Dict[str, torch.Tensor]:
+    """The seven matrices and two norm gains of one decoder layer (same values as in make_weights)."""
+    dt = _TORCH_DTYPE[shape.dtype]
+    d, f = shape.d_model, shape.d_ffn
+    dims = [(d, d), (d, d), (d, d), (d, d), (f, d), (f, d), (d, f)]
+    out: Dict[str, torch.Tensor] = {}
+    for j, (n, (r, c)) in enumerate(zip(_LAYER_NAMES, dims)):
+        out[n] = normal(seed, _S_LAYER0 + layer * _S_PER_LAYER + j, r * c, std, device).view(r, c).to(dt)
+    out["norm_attn"] = torch.ones(d, dtype=dt, device=device)
+    out["norm_ffn"] = torch.ones(d, dtype=dt, device=device)
+    return out
+
+
 def make_weights(shape: ModelShape, seed: int = 0, device="cpu", std: float = 0.02
                  ) -> Dict[str, object]:
     """All tensors of a random-init decoder, canonical [out, in] row-major.
@@ -118,7 +135,7 @@ def make_weights(shape: ModelShape, seed: int = 0, device="cpu", std: float = 0.
     dtype; norm gains are exactly 1.
     """
     dt = _TORCH_DTYPE[shape.dtype]
-    d, f, v = shape.d_model, shape.d_ffn, shape.vocab
+    d, v = shape.d_model, shape.vocab
 
     def mat(stream, rows, cols):
         return normal(seed, stream, rows * cols, std, device).view(rows, cols).to(dt)
@@ -129,15 +146,11 @@ def make_weights(shape: ModelShape, seed: int = 0, device="cpu", std: float = 0.
         "lm_head": mat(_S_LM, v, d),
         "final_norm": torch.ones(d, dtype=dt, device=device),
     }
-    names = ["wq", "wk", "wv", "wo", "wg", "wu", "wd"]
-    dims = [(d, d), (d, d), (d, d), (d, d), (f, d), (f, d), (d, f)]
-    for n in names + ["norm_attn", "norm_ffn"]:
+    for n in _LAYER_NAMES + ["norm_attn", "norm_ffn"]:
         w[n] = []
     for l in range(shape.n_layers):
-        for j, (n, (r, c)) in enumerate(zip(names, dims)):
-            w[n].append(mat(_S_LAYER0 + l * _S_PER_LAYER + j, r, c))
-        w["norm_attn"].append(torch.ones(d, dtype=dt, device=device))
-        w["norm_ffn"].append(torch.ones(d, dtype=dt, device=device))
+        for n, t in make_layer_weights(shape, l, seed, device, std).items():
+            w[n].append(t)
     return w
 
 
