@@ -55,6 +55,8 @@ struct GemmParams {
     int packed;                    // 1: the weight maps are over the packed copy [tile][k-block][box rows][64]
                                    // (see k_pack_weight): a box is addressed by its number, not by row and column
     int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
+    int has_lo;                    // 1: token row r is B row r (bf16 hi part) + B row rh + r (lo part), R <= rh;
+                                   // 0: npad plain bf16 rows (prompt chunks of up to 256 tokens), R <= npad
     int stages;
     int epi;
     int n_out;                     // output features in total
@@ -62,7 +64,7 @@ struct GemmParams {
     float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: rh == 16 (9..16 rows)
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
-    // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kMaxRows]
+    // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kRowsCap]
     const float* sumsq_in;
     int n_parts_in;
     float inv_d_in, eps;
@@ -82,7 +84,7 @@ struct GemmParams {
     const __nv_bfloat16* gain_next;
     __nv_bfloat16* xn_out;         // [2*rh_out.. rows][d]: hi rows then lo rows
     int xn_lo_row0;                // first lo row of xn_out / act_out
-    float* sumsq_out;              // [n_tiles][kMaxRows]
+    float* sumsq_out;              // [n_tiles][kRowsCap]
     // kEpiSwiGLU
     __nv_bfloat16* act_out;        // [rows][f]
 };
@@ -281,9 +283,9 @@ __host__ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, i
 // that the 1 + 2k rows of k = 4 look-ahead tokens go through in one pass).
 struct EpiCtx {
     int lane_in_tile;        // 0..127
-    float* s_rstd;           // [kMaxRows]
+    float* s_rstd;           // [kRowsCap]
     float* s_x;              // [128][9] exchange buffer
-    const unsigned long long* s_kvoff;   // [kMaxRows] cache offset of head 0, feature 0 of each token row (kEpiQKV)
+    const unsigned long long* s_kvoff;   // [kRowsCap] cache offset of head 0, feature 0 of each token row (kEpiQKV)
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -355,7 +357,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
                 __nv_bfloat16 hi, lo;
                 split_bf16(hn * g, hi, lo);
                 p.xn_out[(size_t)r * d + n] = hi;
-                p.xn_out[(size_t)(p.xn_lo_row0 + r) * d + n] = lo;
+                if (p.has_lo) p.xn_out[(size_t)(p.xn_lo_row0 + r) * d + n] = lo;
             }
             ss[j] = hn * hn;
         }
@@ -373,7 +375,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         }
         epi_bar();
         if (L < NR && c0 + L < p.R)
-            p.sumsq_out[(size_t)tile * kMaxRows + c0 + L] =
+            p.sumsq_out[(size_t)tile * kRowsCap + c0 + L] =
                 ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
     } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
         // Both halves of the threads work after the exchange: a gate lane finishes the even rows of its
@@ -395,7 +397,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
                     __nv_bfloat16 hi, lo;
                     split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
                     p.act_out[(size_t)r * p.n_out + n] = hi;
-                    p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
+                    if (p.has_lo) p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
                 }
             }
         }
@@ -552,8 +554,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_epi_done;
     __shared__ int s_last;
     __shared__ int s_epi_fail;
-    __shared__ float s_rstd[kMaxRows];
-    __shared__ unsigned long long s_kvoff[kMaxRows];
+    __shared__ float s_rstd[kRowsCap];
+    __shared__ unsigned long long s_kvoff[kRowsCap];
     __shared__ float s_x[128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
@@ -753,7 +755,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
 #pragma unroll
                         for (int u = 0; u < 4; u++) {
                             const int t = t0 + u * 8 + l8;
-                            if (t < p.n_parts_in) part[u] += __ldcg(p.sumsq_in + (size_t)t * kMaxRows + r);
+                            if (t < p.n_parts_in) part[u] += __ldcg(p.sumsq_in + (size_t)t * kRowsCap + r);
                         }
                     }
                     ss = (part[0] + part[1]) + (part[2] + part[3]);
@@ -768,7 +770,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 }
             }
             epi_bar();
-            const size_t slot_floats = (size_t)p.rh * kTileN;
+            const int rows_acc = p.has_lo ? p.rh : p.npad;          // token rows held by an accumulator
+            const size_t slot_floats = (size_t)rows_acc * kTileN;
             const bool signal = oi + 1 < cp.n_ops;   // a later GEMM of the chain waits for this one's tiles
             for (int it = 0; ok && fetch_piece(oi, it, pc); it++, pidx++) {
                 const int buf = pidx & 1;
@@ -776,7 +779,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
                 float2 cs_pre[16] = {};
-                const bool pre = p.rh == 16 && pc.index == 0;
+                const bool pre = p.rh == 16 && p.has_lo && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
@@ -794,7 +797,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 if (et == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
                 const bool whole = pc.n_pieces == 1;
-                const bool ll = p.rh == 16;                    // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
+                const bool ll = p.rh == 16 && p.has_lo;        // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
                 float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
                 int ll_n = 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
@@ -856,13 +859,15 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     }
                 } else {
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
-                for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                for (int c0 = 0; c0 < rows_acc; c0 += 8) {
                     float hi[8], lo[8];
                     tmem_ld8(t_addr + c0, hi);
-                    tmem_ld8(t_addr + p.rh + c0, lo);
+                    if (p.has_lo) tmem_ld8(t_addr + p.rh + c0, lo);
                     tmem_ld_wait();
+                    if (p.has_lo) {
 #pragma unroll
-                    for (int j = 0; j < 8; j++) hi[j] += lo[j];
+                        for (int j = 0; j < 8; j++) hi[j] += lo[j];
+                    }
                     if (whole) {
                         epi_store<8>(p, ec, pc.tile, c0, hi);
                     } else {
@@ -899,7 +904,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         tile_done = true;
                         const int c_first = cta - pc.index;
                         const int slot_first = pc.first_slot;
-                        for (int c0 = 0; c0 < p.rh; c0 += 8) {
+                        for (int c0 = 0; c0 < rows_acc; c0 += 8) {
                             float acc[8];
 #pragma unroll
                             for (int j = 0; j < 8; j++) acc[j] = 0.f;

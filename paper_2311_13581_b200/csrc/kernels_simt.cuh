@@ -271,12 +271,12 @@ k_split_norm_input(const float* __restrict__ h, const __nv_bfloat16* __restrict_
         const float x = v * __bfloat162float(g[n]);
         const __nv_bfloat16 hi = __float2bfloat16_rn(x);
         xn[(size_t)r * d + n] = hi;
-        xn[(size_t)(lo_row0 + r) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));
+        if (lo_row0 >= 0) xn[(size_t)(lo_row0 + r) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));   // < 0: plain bf16 rows
         const float ss = warp_sum(v * v);
         __syncthreads();
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
         __syncthreads();
-        if (threadIdx.x == 0) sumsq[(size_t)t * kMaxRows + r] = red[0] + red[1] + red[2] + red[3];
+        if (threadIdx.x == 0) sumsq[(size_t)t * kRowsCap + r] = red[0] + red[1] + red[2] + red[3];
     }
 }
 
@@ -327,7 +327,7 @@ k_step_input(const __nv_bfloat16* __restrict__ tok_emb, const __nv_bfloat16* __r
     __syncthreads();
     if (threadIdx.x < 8) {
         const int j = threadIdx.x >> 1, w0 = (threadIdx.x & 1) * 4, t = chunk * 8 + threadIdx.x;
-        if (t * 128 < d) sumsq[(size_t)t * kMaxRows + r] = red[j][w0] + red[j][w0 + 1] + red[j][w0 + 2] + red[j][w0 + 3];
+        if (t * 128 < d) sumsq[(size_t)t * kRowsCap + r] = red[j][w0] + red[j][w0 + 1] + red[j][w0 + 2] + red[j][w0 + 3];
     }
     if (chunk == 0) {
         const int pos = st.kv_len + i;
