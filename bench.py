@@ -54,6 +54,9 @@ WORKLOADS = {
     "7b-k2-ctx2048-T0.8": dict(shape="7b", k=2, prompt=2048, T=0.8, batch=1),
     "7b-k6-ctx2048-T0.8": dict(shape="7b", k=6, prompt=2048, T=0.8, batch=1),
     "7b-k8-ctx2048-T0.8": dict(shape="7b", k=8, prompt=2048, T=0.8, batch=1),
+    # the prompt pass by itself (what comes before the first step): prompt tokens per second
+    "7b-prefill-2048": dict(shape="7b", k=4, prompt=2048, T=0.0, batch=1, prefill=True),
+    "7b-prefill-8192": dict(shape="7b", k=4, prompt=8192, T=0.0, batch=1, prefill=True),
 }
 
 
@@ -294,6 +297,59 @@ def timed_steps(ctx, stream, k, T, u_dev, s0, n_steps, barrier, sampler_gpu=None
     return evs[0].elapsed_time(evs[-1]), per, clocks, s
 
 
+def run_prefill_bench(args, wl, shape):
+    """The prompt pass (pass_prefill) by itself: a step is one prompt of the workload's length through all
+    layers.  Tensor-pipe bound: flops = 2 x tokens x GEMM weights + causal attention, against the sustained
+    bf16 GEMM peak."""
+    import paper_2311_13581_b200 as pb
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    P = wl["prompt"]
+    w = si.make_weights(shape, seed=0, device=dev)
+    ctx = pb.PassContext(shape, w, 1, P + 64, device=dev)
+    prompts = [si.make_prompt(shape, P, seq=i) for i in range(4)]
+    stream = ctx.stream
+    for i in range(max(args.warmup, 3)):
+        ctx.prefill(0, prompts[i % 4])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    n = max(1, min(args.steps, 20))
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    t0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        evs[0].record(stream)
+        for i in range(n):
+            ctx.prefill(0, prompts[i % 4])          # tokens come from host memory; the call synchronises
+            evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    clocks = sampler.stop()
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+    ms = evs[0].elapsed_time(evs[-1]) / n
+    T = P - 1                                          # rows that go through the layers
+    d, f, L = shape.d_model, shape.d_ffn, shape.n_layers
+    gemm_flops = 2.0 * T * L * (4 * d * d + 3 * d * f)
+    attn_flops = 4.0 * (T * (T + 1) / 2) * d * L      # QK^T and PV over the causal triangle
+    pk, pk_kind = peaks()
+    peak = pk.get("bf16_tflops_sustained", pk.get("bf16_tflops"))
+    ach = (gemm_flops + attn_flops) / (ms * 1e-3) / 1e12
+    line = {"metric": "prompt tokens/s through pass_prefill (7B shape, bf16)", "value": T / (ms * 1e-3), "unit": "tok/s",
+            "n_gpus": 1, "steps": n, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype, "data": "synthetic",
+            "config": {"workload": args.workload, "prompt_len": P, "rows": T, "batch": 1,
+                       "l2": "weights of a layer (405 MB) exceed L2; every prompt streams all of them"},
+            "per_step_ms": percentiles(per), "clocks": clocks,
+            "gpu_launches": None,
+            "e2e": {"value": T * n / wall, "unit": "tok/s", "h2d_bytes_per_step": 4 * P, "d2h_bytes_per_step": 0,
+                    "note": "host clock around the same calls (tokens are copied from host memory inside each call)"},
+            "roofline": {"bound": "tensor", "kernel": "pass_prefill: k_gemm_tc_big chains + k_attn_fd (chunk mode)",
+                         "achieved": ach, "peak": peak, "peak_kind": pk_kind + " sustained cuBLAS bf16", "unit": "TFLOP/s",
+                         "frac": ach / peak, "traffic": None, "algorithmic_flops": gemm_flops + attn_flops,
+                         "gemm_flops": gemm_flops, "attention_flops": attn_flops}}
+    print(json.dumps(line))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -309,6 +365,9 @@ def main():
         shape = dataclasses.replace(shape, n_layers=wl["n_layers"])
     if args.impl == "reference":
         run_reference(args, wl, shape)
+        return
+    if wl.get("prefill"):
+        run_prefill_bench(args, wl, shape)
         return
 
     import paper_2311_13581_b200 as pb

@@ -187,6 +187,21 @@ int pass_step_collect(pass_ctx *ctx, int32_t *out_tokens, int32_t *n_out);
 int pass_forward_tokens(pass_ctx *ctx, int seq, const int32_t *tokens, int n,
                         float *logits_out_device, int commit);
 
+/*
+ * Arithmetic of long prompts (bf16 models; the paper names no precision).  A prompt of more than
+ * PASS_MAX_ROWS tokens runs in chunks of up to 1024 (hi + lo) or 2048 (plain) rows as large tensor-core GEMMs
+ * with causal flash attention:
+ *   PASS_PROMPT_HI_LO (default): activations as bf16 hi + lo pairs, the arithmetic of pass_step; the cache
+ *       it leaves agrees with a float64 computation to about 1e-3 per row.
+ *   PASS_PROMPT_BF16: activations, queries and probabilities as single bf16 values - half the tensor-core
+ *       work per token; about 5e-3 per row and layer away from a float64 computation (measured, 7B layer
+ *       shape), which at full depth uses up the 1e-2 bound stated for the logits of later steps.
+ * Host-side setting, applies to later pass_prefill calls.  Errors: INVALID_ARG.
+ */
+#define PASS_PROMPT_HI_LO 0
+#define PASS_PROMPT_BF16  1
+int pass_set_prompt_precision(pass_ctx *ctx, int mode);
+
 /* Forget everything about sequence `seq` (len = 0, no pending token, no drafts). */
 int pass_reset(pass_ctx *ctx, int seq);
 

@@ -20,6 +20,7 @@ PASS_DBG_LOGITS, PASS_DBG_DRAFT_LOGITS, PASS_DBG_KV_LEN, PASS_DBG_N_DRAFT = 0, 1
 PASS_DBG_DRAFTS, PASS_DBG_PENDING, PASS_DBG_N_ACCEPTED, PASS_DBG_STATUS, PASS_DBG_HIDDEN = 4, 5, 6, 7, 8
 PASS_MAX_ROWS = 128
 PASS_HOOK_GEMM_STUCK, PASS_HOOK_ATTN_STALE = 0, 1
+PASS_PROMPT_HI_LO, PASS_PROMPT_BF16 = 0, 1
 PASS_MAX_TOP_K = 1024
 
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
@@ -27,7 +28,7 @@ EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_we
            "pass_set_top_k", "pass_step_two_call", "pass_debug_schedule",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
-           "pass_debug_time_linear", "pass_linear_noalloc", "pass_debug_set"]
+           "pass_debug_time_linear", "pass_linear_noalloc", "pass_debug_set", "pass_set_prompt_precision"]
 
 
 class PassError(RuntimeError):
@@ -86,6 +87,7 @@ def load_library(path: str = LIB_PATH):
     lib.pass_debug_time_linear.argtypes = [vp, ci, ci, ci, vp]
     lib.pass_linear_noalloc.argtypes = [vp, ci, ci, vp, ci, vp]
     lib.pass_debug_set.argtypes = [vp, ci, ci]
+    lib.pass_set_prompt_precision.argtypes = [vp, ci]
     lib.pass_stream.restype = vp
     lib.pass_stream.argtypes = [vp]
     lib.pass_destroy.restype = None
@@ -268,6 +270,10 @@ class PassContext:
         assert y.is_cuda and y.is_contiguous() and y.dtype == self.torch.float32
         _check(self.lib, self.lib.pass_linear_noalloc(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
         return y
+
+    def set_prompt_precision(self, mode: int) -> None:
+        """pass_set_prompt_precision: PASS_PROMPT_HI_LO (default) or PASS_PROMPT_BF16 for long prompts."""
+        _check(self.lib, self.lib.pass_set_prompt_precision(self.h, mode))
 
     def debug_set(self, hook: int, value: int) -> None:
         """pass_debug_set: per-context switches for the tests of the library's error handling."""

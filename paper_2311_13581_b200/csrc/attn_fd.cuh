@@ -34,8 +34,12 @@ struct AttnParams {
     float* part_ml;                // [B][H][n_split][32][2]
     int* counters;                 // [B*H], zero between launches
     __nv_bfloat16* out;            // [rows][d] hi parts, lo parts lo_row0 rows further down
-    int lo_row0;
+    int lo_row0;                   // < 0: plain bf16 output rows, no lo parts
     int debug_stale;               // test hook: the early part pretends the tables said len - debug_stale
+    int out_tile_rows;             // > 0: output rows are laid out in token tiles of this many rows, hi rows of a tile
+                                   // followed by its lo rows (the layout the next GEMM of a prompt chunk reads)
+    int rows_per_block;            // 0: blockIdx.y = sequence, M rows each (a decode step).  > 0: ONE sequence of M rows
+                                   // (a prompt chunk), blockIdx.y = block of rows_per_block rows - causal flash attention
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
@@ -116,7 +120,7 @@ __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int r
                     if (sidx < p.n_split) v += vals[e][sidx] * sm_f[sidx * 32 + i];
                 const __nv_bfloat16 hi = __float2bfloat16_rn(v);
                 p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
             }
         }
     }
@@ -141,7 +145,10 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
 }
 
 // 168 registers x 128 threads is what is left on an SM beside the GEMM kernel's CTA (256 x 168).
-template <int DH, int MT, bool CL>
+// MT = m-tiles of 16 rows per CTA (4 warps: MT = 4 gives every warp its own 16 rows and all keys of a block,
+// the usual flash-attention split for many rows).  HL = queries and probabilities as bf16 hi + lo pairs;
+// without it they are single bf16 values (prompt chunks in plain bf16, half the MMAs).
+template <int DH, int MT, bool CL, bool HL = true>
 __global__ void __maxnreg__(168)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
@@ -161,7 +168,9 @@ k_attn_fd(const AttnParams p) {
     const int head = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int mt = warp % MT, part = warp / MT;
-    const int M = p.M, row0 = b * M;
+    // a decode step: rows b*M .. of sequence b; a prompt chunk: rows b*rows_per_block .. of the one sequence
+    const int row0 = p.rows_per_block ? b * p.rows_per_block : b * p.M;
+    const int M = p.rows_per_block ? min(p.rows_per_block, p.M - row0) : p.M;
     // one thread reads the tables for all, so that the whole CTA works from the same pair even if it
     // reads while they are being written
     __shared__ int s_tab[2];
@@ -187,6 +196,9 @@ k_attn_fd(const AttnParams p) {
         vbase = p.vc + kv_index(p.md, p.layer, seq, head, 0);
     };
     slice(s_tab[0], max(0, s_tab[1] - p.debug_stale));
+    // rows of this launch's own chunk ahead of this block are cache rows the awaited kernel writes: in chunk
+    // mode only positions before the chunk's first row may be fetched early
+    const int early_len = p.rows_per_block ? min(len, *(volatile const int*)(p.row_pos)) : len;
     const uint32_t sK = smem_u32(smem_attn), sV = sK + kAttnStages * TILE_BYTES;
 
     auto load_block = [&](int blk) {
@@ -207,7 +219,7 @@ k_attn_fd(const AttnParams p) {
     uint32_t early = 0;
 #pragma unroll
     for (int st = 0; st < kAttnStages; st++) {
-        if (st < nb && min(k_end, k_begin + (st + 1) * kAttnBK) <= len) { load_block(st); early |= 1u << st; }
+        if (st < nb && min(k_end, k_begin + (st + 1) * kAttnBK) <= early_len) { load_block(st); early |= 1u << st; }
     }
     cp_async_commit();
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -287,8 +299,10 @@ k_attn_fd(const AttnParams p) {
                     ldsm_x4(kS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
                     mma_bf16_16816(s[0], qf[ks], r[0], r[1]);
                     mma_bf16_16816(s[1], qf[ks], r[2], r[3]);
-                    mma_bf16_16816(sl[0], qfl[ks], r[0], r[1]);
-                    mma_bf16_16816(sl[1], qfl[ks], r[2], r[3]);
+                    if (HL) {
+                        mma_bf16_16816(sl[0], qfl[ks], r[0], r[1]);
+                        mma_bf16_16816(sl[1], qfl[ks], r[2], r[3]);
+                    }
                 }
 #pragma unroll
                 for (int n = 0; n < 2; n++)
@@ -352,8 +366,10 @@ k_attn_fd(const AttnParams p) {
                     ldsm_x4_trans(vS + (uint32_t)((key * CH + (c ^ (key & 7))) * 16), r);
                     mma_bf16_16816(o[2 * np], pa, r[0], r[1]);
                     mma_bf16_16816(o[2 * np + 1], pa, r[2], r[3]);
-                    mma_bf16_16816(o[2 * np], pl, r[0], r[1]);
-                    mma_bf16_16816(o[2 * np + 1], pl, r[2], r[3]);
+                    if (HL) {
+                        mma_bf16_16816(o[2 * np], pl, r[0], r[1]);
+                        mma_bf16_16816(o[2 * np + 1], pl, r[2], r[3]);
+                    }
                 }
             }
         }
@@ -406,8 +422,10 @@ k_attn_fd(const AttnParams p) {
         if (p.n_split == 1) {
             const float v = acc / ll;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-            p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-            p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            const int g_row = row0 + i;
+            const int o_row = p.out_tile_rows ? (g_row / p.out_tile_rows) * 2 * p.out_tile_rows + g_row % p.out_tile_rows : g_row;
+            p.out[(size_t)o_row * p.md.d + head * DH + dcol] = hi;
+            if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + o_row) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
         } else if (CL) {
             float* cl_o = sm_o + 4 * 16 * DH + 128;          // [32][DH], behind the warp staging area
             float* cl_ml = cl_o + 32 * DH;                   // [32][2]
@@ -450,7 +468,7 @@ k_attn_fd(const AttnParams p) {
             const int dcol = idx % DH;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
             p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-            p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
         cluster_sync_all();                                  // nobody leaves while its memory is still being read
         return;

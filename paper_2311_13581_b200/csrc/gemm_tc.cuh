@@ -38,6 +38,7 @@
 namespace pass {
 
 constexpr int kTileN = 128;
+constexpr int kTokTile = 256;                           // token rows of one accumulator at most (the MMA's N)
 constexpr int kBlockK = 64;
 constexpr int kGemmThreads = 256;
 constexpr int kATileBytes = kTileN * kBlockK * 2;       // 16 KB
@@ -55,6 +56,10 @@ struct GemmParams {
     int packed;                    // 1: the weight maps are over the packed copy [tile][k-block][box rows][64]
                                    // (see k_pack_weight): a box is addressed by its number, not by row and column
     int npad, rh, R;               // B rows (hi | lo halves of rh rows each), live rows
+    int n_tok_tiles;               // > 0 (prompt chunks): the token rows are cut into tiles of npad rows too; unit u of
+                                   // the schedule is (feature tile u / n_tok_tiles, token tile u % n_tok_tiles) and
+                                   // n_tiles counts units.  0: one token tile, unit = feature tile
+    int whole_only;                // 1: every unit is computed whole by one CTA (unit j * CTAs + c), nothing is split
     int has_lo;                    // 1: token row r is B row r (bf16 hi part) + B row rh + r (lo part), R <= rh;
                                    // 0: npad plain bf16 rows (prompt chunks of up to 256 tokens), R <= npad
     int stages;
@@ -236,6 +241,18 @@ __host__ __device__ __forceinline__ int unit_owner(long long x, long long U, lon
 // other CTA: no arrival counter and no trip for partial sums on the path to the next GEMM.  With fewer
 // tiles than CTAs everything is streamed.
 __host__ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, int G, int it, Piece& out) {
+    if (p.whole_only) {
+        // prompt chunks: many large units, each done whole; CTAs that run side by side take neighbouring units,
+        // i.e. the token tiles of the same few feature tiles, so a weight tile leaves HBM once and is then found in L2
+        const long long tile = (long long)it * G + c;
+        if (tile >= p.n_tiles) return false;
+        out.tile = (int)tile;
+        out.kb0 = 0;
+        out.kb1 = p.kb_per_tile;
+        out.n_pieces = 1;
+        out.index = out.slot = out.first_slot = 0;
+        return true;
+    }
     const int rounds = p.n_tiles >= G ? p.n_tiles / G : 0;      // whole tiles per CTA
     const int n_sk = p.n_tiles - rounds * G;                     // tiles that are streamed, [0, n_sk)
     const long long U = (long long)n_sk * p.kb_per_tile;
@@ -283,9 +300,13 @@ __host__ __device__ __forceinline__ bool get_piece(const GemmParams& p, int c, i
 // that the 1 + 2k rows of k = 4 look-ahead tokens go through in one pass).
 struct EpiCtx {
     int lane_in_tile;        // 0..127
-    float* s_rstd;           // [kRowsCap]
+    float* s_rstd;           // [kTokTile]
     float* s_x;              // [128][9] exchange buffer
-    const unsigned long long* s_kvoff;   // [kRowsCap] cache offset of head 0, feature 0 of each token row (kEpiQKV)
+    const unsigned long long* s_kvoff;   // [kTokTile] cache offset of head 0, feature 0 of each token row (kEpiQKV)
+    int row_base;            // first token row of the token tile being finished (0 unless the rows are tiled)
+    int rows_live;           // live rows of that token tile; s_rstd / s_kvoff are indexed by the row within the tile
+    int out_row_base;        // row of xn_out / act_out that holds the tile's first token (its lo part xn_lo_row0 further
+                             // down): token tiles of hi | lo rows are laid out one after another, as the next GEMM reads them
 };
 
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
@@ -307,7 +328,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         if (n < p.n_out) {
 #pragma unroll
             for (int j = 0; j < NR; j++)
-                if (c0 + j < p.R) p.logits[(size_t)(c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
+                if (c0 + j < ec.rows_live) p.logits[(size_t)(ec.row_base + c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
         }
     } else if (p.epi == kEpiQKV) {
         const int d = p.md.d, dh = p.md.dh;
@@ -319,21 +340,21 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const size_t head_off = ((size_t)head * p.md.cap) * dh + i;
 #pragma unroll
         for (int j = 0; j < NR; j++) {
-            const int r = min(c0 + j, p.R - 1);
+            const int r = min(c0 + j, ec.rows_live - 1);
             kvo[j] = (size_t)ec.s_kvoff[r] + head_off;
-            cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)r * (dh / 2) + (i >> 1));
+            cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)(ec.row_base + r) * (dh / 2) + (i >> 1));
         }
 #pragma unroll
         for (int j = 0; j < NR; j++) {
             const int r = c0 + j;
-            const float x = v[j] * (r < p.R ? ec.s_rstd[r] : 0.f);
+            const float x = v[j] * (r < ec.rows_live ? ec.s_rstd[r] : 0.f);
             const float other = __shfl_xor_sync(0xffffffffu, x, 1);
-            if (r < p.R) {
+            if (r < ec.rows_live) {
                 if (which == 2) {
                     p.vc[kvo[j]] = __float2bfloat16_rn(x);
                 } else {
                     const float y = (i & 1) ? other * cs[j].y + x * cs[j].x : x * cs[j].x - other * cs[j].y;
-                    if (which == 0) p.q_out[(size_t)r * d + c] = y;
+                    if (which == 0) p.q_out[(size_t)(ec.row_base + r) * d + c] = y;
                     else p.kc[kvo[j]] = __float2bfloat16_rn(y);
                 }
             }
@@ -346,18 +367,19 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         float ss[NR], hv[NR];
 #pragma unroll
         for (int j = 0; j < NR; j++)      // all loads first: they are independent of the stores below
-            hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < p.R && n < d) ? __ldcg(p.h + (size_t)(c0 + j) * d + n) : 0.f);
+            hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < ec.rows_live && n < d) ? __ldcg(p.h + (size_t)(ec.row_base + c0 + j) * d + n) : 0.f);
 #pragma unroll
         for (int j = 0; j < NR; j++) {
-            const int r = c0 + j;
+            const int r = ec.row_base + c0 + j;
             float hn = 0.f;
-            if (r < p.R && n < d) {
+            if (c0 + j < ec.rows_live && n < d) {
                 hn = hv[j] + v[j];
                 p.h[(size_t)r * d + n] = hn;
                 __nv_bfloat16 hi, lo;
                 split_bf16(hn * g, hi, lo);
-                p.xn_out[(size_t)r * d + n] = hi;
-                if (p.has_lo) p.xn_out[(size_t)(p.xn_lo_row0 + r) * d + n] = lo;
+                const size_t orow = (size_t)(ec.out_row_base + c0 + j);
+                p.xn_out[orow * d + n] = hi;
+                if (p.has_lo) p.xn_out[(orow + p.xn_lo_row0) * d + n] = lo;
             }
             ss[j] = hn * hn;
         }
@@ -374,8 +396,8 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             for (int j = 0; j < NR; j++) ec.s_x[warp_q * NR + j] = ss[j];
         }
         epi_bar();
-        if (L < NR && c0 + L < p.R)
-            p.sumsq_out[(size_t)tile * kRowsCap + c0 + L] =
+        if (L < NR && c0 + L < ec.rows_live)
+            p.sumsq_out[(size_t)tile * kRowsCap + ec.row_base + c0 + L] =
                 ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
     } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
         // Both halves of the threads work after the exchange: a gate lane finishes the even rows of its
@@ -389,15 +411,15 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         if (n < p.n_out) {
 #pragma unroll
             for (int j = 0; j < NR; j++) {
-                const int r = c0 + j;
-                if (r < p.R && ((j & 1) == (L >> 6))) {
-                    const float rs = ec.s_rstd[r];
+                if (c0 + j < ec.rows_live && ((j & 1) == (L >> 6))) {
+                    const float rs = ec.s_rstd[c0 + j];
                     const float mine = v[j] * rs, theirs = ec.s_x[other * 9 + j] * rs;
                     const float g = L < 64 ? mine : theirs, u = L < 64 ? theirs : mine;
                     __nv_bfloat16 hi, lo;
                     split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
-                    p.act_out[(size_t)r * p.n_out + n] = hi;
-                    if (p.has_lo) p.act_out[(size_t)(p.xn_lo_row0 + r) * p.n_out + n] = lo;
+                    const size_t orow = (size_t)(ec.out_row_base + c0 + j);
+                    p.act_out[orow * p.n_out + n] = hi;
+                    if (p.has_lo) p.act_out[(orow + p.xn_lo_row0) * p.n_out + n] = lo;
                 }
             }
         }
@@ -544,8 +566,11 @@ __device__ __forceinline__ void weight_xy(const GemmParams& p, int y_rowmajor, i
     }
 }
 
-__global__ void __maxnreg__(168)
-k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+// BIG = false: the decode step's kernel (hi | lo rows, one token tile).  BIG = true adds what prompt chunks
+// need (token tiles, plain bf16 rows, whole-unit schedule, loads one row group ahead in the epilogue); it is a
+// second instantiation so that the step's kernel keeps its registers.
+template <bool BIG>
+__device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const ChainParams& cp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
     __shared__ uint32_t s_tmem_base;
@@ -554,8 +579,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
     __shared__ int s_epi_done;
     __shared__ int s_last;
     __shared__ int s_epi_fail;
-    __shared__ float s_rstd[kRowsCap];
-    __shared__ unsigned long long s_kvoff[kRowsCap];
+    __shared__ float s_rstd[kTokTile];
+    __shared__ unsigned long long s_kvoff[kTokTile];
     __shared__ float s_x[128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
@@ -633,7 +658,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
-                    weight_box(p, maps.m[oi], pc.tile, 0, m, y);
+                    weight_box(p, maps.m[oi], (BIG && p.n_tok_tiles > 0) ? pc.tile / p.n_tok_tiles : pc.tile, 0, m, y);
                     for (int kb = pc.kb0; kb < pc.kb1; kb++) {
                         const int s = fill % S;
                         const uint32_t parity = ((fill / S) & 1) ^ 1;
@@ -668,7 +693,8 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
-                    weight_box(p, maps.m[oi], pc.tile, 1, m, y);
+                    weight_box(p, maps.m[oi], (BIG && p.n_tok_tiles > 0) ? pc.tile / p.n_tok_tiles : pc.tile, 1, m, y);
+                    const int b_row0 = (BIG && p.n_tok_tiles > 0) ? (pc.tile % p.n_tok_tiles) * p.npad : 0;    // token tile
                     for (int kb = pc.kb0; kb < pc.kb1; kb++) {
                         const int s = fill % S;
                         if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
@@ -681,7 +707,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                         } else {
                             mbar_expect_tx(bar_full + 8 * s, stage_bytes - kATileBytes);
                         }
-                        tma_load_2d(dst + kATileBytes, &maps.m[oi][3], bar_full + 8 * s, kb * kBlockK, 0, pol_x);
+                        tma_load_2d(dst + kATileBytes, &maps.m[oi][3], bar_full + 8 * s, kb * kBlockK, b_row0, pol_x);
                         fill++;
                         *(volatile int*)&s_issued_b = fill;
                     }
@@ -746,31 +772,40 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
             // rstd of the input rows: eight lanes per row, each sums every eighth part (its loads are
             // independent, so a row costs one trip to L2 whatever the number of parts), then a fixed-order
             // butterfly.  The first accumulator of a short first piece may already be waiting for us.
-            for (int r0 = 0; r0 < p.R; r0 += 16) {
-                const int r = r0 + (et >> 3), l8 = et & 7;
-                float ss = 0.f;
-                if (p.sumsq_in && r < p.R) {
-                    float part[4] = {0.f, 0.f, 0.f, 0.f};
-                    for (int t0 = 0; t0 < p.n_parts_in; t0 += 32) {
+            // (rows of the token tile that starts at row `base`; the tables are indexed by the row within the tile)
+            auto fill_row_tables = [&](int base, int n_rows) {
+                for (int r0 = 0; r0 < n_rows; r0 += 16) {
+                    const int lr = r0 + (et >> 3), r = base + lr, l8 = et & 7;
+                    float ss = 0.f;
+                    if (p.sumsq_in && lr < n_rows) {
+                        float part[4] = {0.f, 0.f, 0.f, 0.f};
+                        for (int t0 = 0; t0 < p.n_parts_in; t0 += 32) {
 #pragma unroll
-                        for (int u = 0; u < 4; u++) {
-                            const int t = t0 + u * 8 + l8;
-                            if (t < p.n_parts_in) part[u] += __ldcg(p.sumsq_in + (size_t)t * kRowsCap + r);
+                            for (int u = 0; u < 4; u++) {
+                                const int t = t0 + u * 8 + l8;
+                                if (t < p.n_parts_in) part[u] += __ldcg(p.sumsq_in + (size_t)t * kRowsCap + r);
+                            }
                         }
+                        ss = (part[0] + part[1]) + (part[2] + part[3]);
                     }
-                    ss = (part[0] + part[1]) + (part[2] + part[3]);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+                    if (lr < n_rows && l8 == 0) {
+                        s_rstd[lr] = p.sumsq_in ? rsqrtf(ss * p.inv_d_in + p.eps) : 1.f;
+                        if (p.epi == kEpiQKV)
+                            s_kvoff[lr] = kv_index(p.md, p.layer, __ldg(p.row_seq + r), 0, __ldg(p.row_pos + r));
+                    }
                 }
-                ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-                ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-                ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-                if (r < p.R && l8 == 0) {
-                    s_rstd[r] = p.sumsq_in ? rsqrtf(ss * p.inv_d_in + p.eps) : 1.f;
-                    if (p.epi == kEpiQKV)
-                        s_kvoff[r] = kv_index(p.md, p.layer, __ldg(p.row_seq + r), 0, __ldg(p.row_pos + r));
-                }
-            }
+            };
+            int cur_tt = -1;
+            ec.row_base = 0;
+            ec.out_row_base = 0;
+            ec.rows_live = p.R;
+            if (!BIG || p.n_tok_tiles == 0) fill_row_tables(0, p.R);
             epi_bar();
-            const int rows_acc = p.has_lo ? p.rh : p.npad;          // token rows held by an accumulator
+            const bool has_lo = !BIG || p.has_lo;
+            const int rows_acc = has_lo ? p.rh : p.npad;            // token rows held by an accumulator
             const size_t slot_floats = (size_t)rows_acc * kTileN;
             const bool signal = oi + 1 < cp.n_ops;   // a later GEMM of the chain waits for this one's tiles
             for (int it = 0; ok && fetch_piece(oi, it, pc); it++, pidx++) {
@@ -779,7 +814,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
                 float2 cs_pre[16] = {};
-                const bool pre = p.rh == 16 && p.has_lo && pc.index == 0;
+                const bool pre = p.rh == 16 && has_lo && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
@@ -790,6 +825,20 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     for (int j = 0; j < 16; j++)
                         cs_pre[j] = __ldg(p.rope_cs + (size_t)min(j, p.R - 1) * (p.md.dh / 2) + i2);
                 }
+                int ftile = pc.tile;                           // feature tile of this piece
+                if (BIG && p.n_tok_tiles > 0) {
+                    ftile = pc.tile / p.n_tok_tiles;
+                    const int tt = pc.tile % p.n_tok_tiles;
+                    if (tt != cur_tt) {                        // another token tile: its rows' factors and cache offsets
+                        epi_bar();
+                        const int tile_tokens = p.has_lo ? p.rh : p.npad;
+                        ec.row_base = tt * tile_tokens;
+                        ec.out_row_base = tt * p.npad;
+                        ec.rows_live = min(tile_tokens, p.R - ec.row_base);
+                        fill_row_tables(ec.row_base, ec.rows_live);
+                        cur_tt = tt;
+                    }
+                }
                 // each thread waits for itself; the outcome is made uniform before any barrier is used
                 if (!mbar_wait(bar_accf + 8 * buf, (pidx >> 1) & 1, &s_abort, cp.status)) *(volatile int*)&s_epi_fail = 1;
                 epi_bar();
@@ -797,7 +846,7 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                 if (et == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
                 const bool whole = pc.n_pieces == 1;
-                const bool ll = p.rh == 16 && p.has_lo;        // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
+                const bool ll = p.rh == 16 && has_lo;          // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
                 float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
                 int ll_n = 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
@@ -859,17 +908,38 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
                     }
                 } else {
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
+                // Whole tiles of many rows (prompt chunks): what the residual epilogue reads is requested one
+                // group of eight rows ahead, so that a group does not begin with a trip to L2.
+                const bool ahead = BIG && whole && p.epi == kEpiResid;
+                const int n_res = ftile * kTileN + ec.lane_in_tile;
+                float g_res = 0.f, hv_cur[8], hv_nxt[8];
+                auto load_h = [&](int c0, float (&hv)[8]) {
+#pragma unroll
+                    for (int j = 0; j < 8; j++)
+                        hv[j] = (c0 + j < ec.rows_live && n_res < p.n_out)
+                                    ? __ldcg(p.h + (size_t)(ec.row_base + c0 + j) * p.n_out + n_res) : 0.f;
+                };
+                if (ahead) {
+                    g_res = n_res < p.n_out ? __bfloat162float(p.gain_next[n_res]) : 0.f;
+                    load_h(0, hv_cur);
+                }
                 for (int c0 = 0; c0 < rows_acc; c0 += 8) {
+                    if (whole && c0 >= ec.rows_live) break;        // rows beyond the live ones: nothing to write
                     float hi[8], lo[8];
                     tmem_ld8(t_addr + c0, hi);
-                    if (p.has_lo) tmem_ld8(t_addr + p.rh + c0, lo);
+                    if (has_lo) tmem_ld8(t_addr + p.rh + c0, lo);
+                    if (ahead) load_h(c0 + 8, hv_nxt);
                     tmem_ld_wait();
-                    if (p.has_lo) {
+                    if (has_lo) {
 #pragma unroll
                         for (int j = 0; j < 8; j++) hi[j] += lo[j];
                     }
                     if (whole) {
-                        epi_store<8>(p, ec, pc.tile, c0, hi);
+                        epi_store<8>(p, ec, ftile, c0, hi, ahead ? hv_cur : nullptr, ahead ? &g_res : nullptr);
+                        if (ahead) {
+#pragma unroll
+                            for (int j = 0; j < 8; j++) hv_cur[j] = hv_nxt[j];
+                        }
                     } else {
                         // partial slot layout [rh/4][feature] of float4 (four token rows of one feature): a warp
                         // stores and loads 512 contiguous bytes per instruction
@@ -969,6 +1039,16 @@ k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainP
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
     }
+}
+
+__global__ void __maxnreg__(168)
+k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    gemm_chain_body<false>(maps, cp);
+}
+// prompt chunks: alone on its SM (192 KB of ring), so the register cap of the step's kernel does not apply
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc_big(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    gemm_chain_body<true>(maps, cp);
 }
 
 }  // namespace pass

@@ -262,16 +262,18 @@ k_attn_simple(const float* __restrict__ qbuf, int ldq, const int* __restrict__ r
 // rows; sumsq[t][r] = sum of h^2 over features 128t .. 128t+127.
 __global__ void __launch_bounds__(128)
 k_split_norm_input(const float* __restrict__ h, const __nv_bfloat16* __restrict__ g, int d,
-                   __nv_bfloat16* __restrict__ xn, int lo_row0, float* __restrict__ sumsq) {
+                   __nv_bfloat16* __restrict__ xn, int lo_row0, float* __restrict__ sumsq, int tile_rows) {
     __shared__ float red[4];
     const int r = blockIdx.x;
+    // tile_rows > 0: token tiles of tile_rows hi rows followed by their lo rows (prompt chunks with hi + lo parts)
+    const int xr = tile_rows ? (r / tile_rows) * 2 * tile_rows + r % tile_rows : r;
     for (int t = 0; t < d / 128; t++) {
         const int n = t * 128 + threadIdx.x;
         const float v = h[(size_t)r * d + n];
         const float x = v * __bfloat162float(g[n]);
         const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-        xn[(size_t)r * d + n] = hi;
-        if (lo_row0 >= 0) xn[(size_t)(lo_row0 + r) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));   // < 0: plain bf16 rows
+        xn[(size_t)xr * d + n] = hi;
+        if (lo_row0 >= 0) xn[(size_t)(lo_row0 + xr) * d + n] = __float2bfloat16_rn(x - __bfloat162float(hi));   // < 0: plain bf16 rows
         const float ss = warp_sum(v * v);
         __syncthreads();
         if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;

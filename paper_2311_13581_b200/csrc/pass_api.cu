@@ -66,16 +66,18 @@ Layout make_layout(const pass_config& c) {
     Layout L;
     Carve cv;
     const size_t R = kMaxRows, d = c.d_model, f = c.d_ffn, V = c.vocab, B = c.max_batch;
+    // rows of one launch: a prompt chunk of a bf16 model has up to kRowsCap, everything else up to kMaxRows
+    const size_t RC = c.dtype == PASS_DTYPE_BF16 ? kRowsCap : kMaxRows;
     L.states = cv.take(B * sizeof(SeqState));
     L.params = cv.take(sizeof(StepParams));
     L.unif = cv.take(B * kUSlots * sizeof(float));
     L.status = cv.take(sizeof(int));
-    L.row_seq = cv.take(R * sizeof(int));
-    L.row_pos = cv.take(R * sizeof(int));
-    L.tok = cv.take(R * sizeof(int));
-    L.cs = cv.take(R * (c.d_head / 2) * sizeof(float2));
+    L.row_seq = cv.take(RC * sizeof(int));
+    L.row_pos = cv.take(RC * sizeof(int));
+    L.tok = cv.take(RC * sizeof(int));
+    L.cs = cv.take(RC * (c.d_head / 2) * sizeof(float2));
     L.invfreq = cv.take((c.d_head / 2) * sizeof(double));
-    L.h = cv.take(R * d * 4);
+    L.h = cv.take(RC * d * 4);
     L.xn = cv.take(R * d * 4);
     L.qkv = cv.take(R * 3 * d * 4);
     L.attn = cv.take(R * d * 4);
@@ -96,12 +98,12 @@ Layout make_layout(const pass_config& c) {
     L.attn_po = L.attn_pml = L.attn_cnt = L.chain_flags = 0;
     L.packed = L.packed_bytes = 0;
     if (c.dtype == PASS_DTYPE_BF16) {
-        L.xn_bf = cv.take(2 * R * d * 2);
-        L.attn_bf = cv.take(2 * R * d * 2);
-        L.act_bf = cv.take(2 * R * f * 2);
-        L.q_out = cv.take(R * d * 4);
-        L.sumsq_a = cv.take((d / 128 + 1) * R * 4);
-        L.sumsq_b = cv.take((d / 128 + 1) * R * 4);
+        L.xn_bf = cv.take(RC * d * 2);           // kRowsCap plain rows, or hi rows + lo rows of a step
+        L.attn_bf = cv.take(RC * d * 2);
+        L.act_bf = cv.take(RC * f * 2);
+        L.q_out = cv.take(RC * d * 4);
+        L.sumsq_a = cv.take((d / 128 + 1) * RC * 4);
+        L.sumsq_b = cv.take((d / 128 + 1) * RC * 4);
         L.partial_ws = cv.take((size_t)kMaxOps * kMaxCtas * 2 * R * kTileN * 4);
         L.counters = cv.take(4096 * 4);
         L.ll_ws = cv.take(kLLRegionBytes * kMaxOps);
@@ -155,11 +157,12 @@ struct pass_ctx {
     int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
     // Function attributes and occupancy answers belong to the device the context lives on, so they are
     // remembered per context, never per process.
-    size_t gemm_smem_set = 0;
+    size_t gemm_smem_set = 0, gemm_big_smem_set = 0;
     std::map<int, bool> attn_attr_set;         // by kernel instance
     std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
     bool use_tc = false;
+    bool prompt_plain_bf16 = false;    // pass_set_prompt_precision: long prompts with plain bf16 activations
     bool packed = false;               // the GEMMs stream the packed copy of the weights (PASS_NO_PACK: the caller's matrices)
     char* d_packed = nullptr;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
@@ -323,9 +326,9 @@ static const pass_ctx::BMaps* get_bmaps(pass_ctx* c, int npad) {
     auto it = c->bmaps.find(npad);
     if (it != c->bmaps.end()) return &it->second;
     pass_ctx::BMaps bm;
-    if (!make_map(&bm.xn, c->d_xn_bf, 2 * kMaxRows, c->md.d, npad)) return nullptr;
-    if (!make_map(&bm.attn, c->d_attn_bf, 2 * kMaxRows, c->md.d, npad)) return nullptr;
-    if (!make_map(&bm.act, c->d_act_bf, 2 * kMaxRows, c->md.f, npad)) return nullptr;
+    if (!make_map(&bm.xn, c->d_xn_bf, kRowsCap, c->md.d, npad)) return nullptr;
+    if (!make_map(&bm.attn, c->d_attn_bf, kRowsCap, c->md.d, npad)) return nullptr;
+    if (!make_map(&bm.act, c->d_act_bf, kRowsCap, c->md.f, npad)) return nullptr;
     return &(c->bmaps[npad] = bm);
 }
 
@@ -349,6 +352,7 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     p.md = c->md;
     p.xn_lo_row0 = npad / 2;
     p.packed = c->packed ? 1 : 0;
+    p.has_lo = 1;
     return p;
 }
 
@@ -402,12 +406,15 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     for (int j = n_ops; j < kMaxOps; j++)
         for (int q = 0; q < 4; q++) maps.m[j][q] = ops[0].a0;
     const size_t smem = (size_t)cp.stages * (kATileBytes + cp.npad * 128) + 1024;
-    if (smem > c->gemm_smem_set) {
-        note_err(c, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "k_gemm_tc shared memory size");
+    const bool big = ops[0].p.whole_only != 0;        // a prompt chunk: the kernel instance with token tiles
+    auto kern = big ? k_gemm_tc_big : k_gemm_tc;
+    size_t& smem_set = big ? c->gemm_big_smem_set : c->gemm_smem_set;
+    if (smem > smem_set) {
+        note_err(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "k_gemm_tc shared memory size");
         // all of the SM's L1/shared storage as shared memory: lets the CTA of the next launch become
         // resident (and start pulling weights) while this launch's CTA is still running
-        note_err(c, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_gemm_tc carveout");
-        c->gemm_smem_set = smem;
+        note_err(c, cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_gemm_tc carveout");
+        smem_set = smem;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -423,7 +430,7 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = c->use_pdl ? 1 : 0;
-    note_err(c, cudaLaunchKernelEx(&cfg, k_gemm_tc, maps, cp), "k_gemm_tc launch");
+    note_err(c, cudaLaunchKernelEx(&cfg, kern, maps, cp), "k_gemm_tc launch");
     c->launches++;
 }
 
@@ -511,7 +518,16 @@ static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
 }
 
 // GEMMs of the decoder layers as chain entries.
-static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l) {
+// Prompt chunks (big): the rows are plain bf16, cut into token tiles of 256 rows; every (feature tile, token
+// tile) unit is computed whole by one CTA.
+static void set_big(pass_ctx* c, GemmParams& p, int R, int feat_tiles) {
+    p.has_lo = c->prompt_plain_bf16 ? 0 : 1;
+    p.whole_only = 1;
+    const int tile_tokens = p.has_lo ? kTokTile / 2 : kTokTile;     // hi | lo rows: 128 tokens fill the MMA's 256 columns
+    p.n_tok_tiles = (R + tile_tokens - 1) / tile_tokens;
+    p.n_tiles = feat_tiles * p.n_tok_tiles;
+}
+static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l, bool big) {
     typedef __nv_bfloat16 bf;
     const int d = c->md.d, dt = d / kTileN;
     ChainOp o;
@@ -521,11 +537,13 @@ static ChainOp op_qkv(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, i
     o.p.q_out = c->d_q_out; o.p.rope_cs = c->d_cs; o.p.row_seq = c->d_row_seq; o.p.row_pos = c->d_row_pos;
     o.p.layer = l; o.p.kc = (bf*)c->kv_k; o.p.vc = (bf*)c->kv_v;
     o.a0 = c->tm_wq[l]; o.a1 = c->tm_wk[l]; o.a2 = c->tm_wv[l]; o.b = bm->xn;
+    if (big) set_big(c, o.p, R, 3 * dt);
     return o;
 }
 // O-projection -> gate|up -> down of layer l, then the next layer's QKV, or the output head (head = true)
 // after the last layer, or nothing.  Returns the number of entries written.
-static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l, bool head, ChainOp* ch) {
+static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps* bm, int l, bool head, ChainOp* ch,
+                             bool big = false) {
     typedef __nv_bfloat16 bf;
     const ModelDims& md = c->md;
     const int d = md.d, f = md.f, dt = d / kTileN;
@@ -535,6 +553,7 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
         o.p.h = c->d_h; o.p.gain_next = (const bf*)c->norm_ffn[l]; o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_b;
         o.a0 = o.a1 = o.a2 = c->tm_wo[l]; o.b = bm->attn;
+        if (big) set_big(c, o.p, R, dt);
     }
     {   // gate | up, interleaved by 64 rows, SwiGLU in the epilogue
         ChainOp& o = ch[n++];
@@ -543,6 +562,7 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p.sumsq_in = c->d_sumsq_b; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
         o.p.act_out = c->d_act_bf;
         o.a0 = c->tm_wg[l]; o.a1 = o.a2 = c->tm_wu[l]; o.b = bm->xn;
+        if (big) set_big(c, o.p, R, (f + 63) / 64);
     }
     {   // down projection + residual; prepares the input of the next norm
         ChainOp& o = ch[n++];
@@ -551,15 +571,17 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p.gain_next = (const bf*)(l + 1 < md.n_layers ? c->norm_attn[l + 1] : c->final_norm);
         o.p.xn_out = c->d_xn_bf; o.p.sumsq_out = c->d_sumsq_a;
         o.a0 = o.a1 = o.a2 = c->tm_wd[l]; o.b = bm->act;
+        if (big) set_big(c, o.p, R, dt);
     }
     if (l + 1 < md.n_layers) {
-        ch[n++] = op_qkv(c, R, npad, bm, l + 1);
+        ch[n++] = op_qkv(c, R, npad, bm, l + 1, big);
     } else if (head) {
         ChainOp& o = ch[n++];
         o.p = gemm_base(c, R, npad, d, (md.V + kTileN - 1) / kTileN, md.V, kEpiLogits);
         o.p.sumsq_in = c->d_sumsq_a; o.p.n_parts_in = dt; o.p.inv_d_in = 1.f / d;
         o.p.logits = c->d_logits;
         o.a0 = o.a1 = o.a2 = c->tm_lm; o.b = bm->xn;
+        if (big) set_big(c, o.p, R, (md.V + kTileN - 1) / kTileN);
     }
     return n;
 }
@@ -569,45 +591,78 @@ static void launch_ops(pass_ctx* c, ChainOp* ch, int n) {
     else launch_chain(c, ch, n);
 }
 
+// Rows of ONE sequence as a prompt chunk: causal flash attention, a CTA per head and block of 64 rows.
+template <int DH, bool HL>
+static void launch_attn_chunk(pass_ctx* c, AttnParams ap) {
+    ap.n_split = 1;
+    ap.rows_per_block = 64;
+    constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
+    bool& set = c->attn_attr_set[DH * 8 + 4 * 2 + (HL ? 64 : 32)];
+    if (!set) {
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, 4, false, HL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->md.H, (ap.M + 63) / 64, 1);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, 4, false, HL>, ap), "k_attn_fd (chunk) launch");
+    c->launches++;
+}
+
 // R rows = n_seq sequences x M rows each (M = R when n_seq == 1).
 // input_ready: the rotary table and the first layer's norm input have been produced already (k_step_input).
-static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool input_ready = false) {
+// big: a prompt chunk of up to kRowsCap rows of one sequence in plain bf16 (see set_big).
+static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool input_ready = false, bool big = false) {
     const ModelDims& md = c->md;
-    const int d = md.d, npad = npad_for(R), rh = npad / 2;
+    const int d = md.d, npad = big ? kTokTile : npad_for(R), rh = npad / 2;
     const pass_ctx::BMaps* bm = get_bmaps(c, npad);
     if (!bm) return PASS_ERR_CUDA;
     typedef __nv_bfloat16 bf;
     chain_counters_clear(c);
     if (!input_ready) {
         LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
-        LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, rh, c->d_sumsq_a);
+        const bool plain = big && c->prompt_plain_bf16;
+        LAUNCH(c, k_split_norm_input, R, 128, c->d_h, (const bf*)c->norm_attn[0], d, c->d_xn_bf, plain ? -1 : rh, c->d_sumsq_a,
+               big && !plain ? rh : 0);
     }
     ChainOp chain[kMaxOps];
     // Kernels of a step: QKV_0 | per layer: attention, then ONE launch running
     // O-projection -> gate|up -> down -> (next layer's QKV, or the output head after the last layer).
-    chain[0] = op_qkv(c, R, npad, bm, 0);
+    chain[0] = op_qkv(c, R, npad, bm, 0, big);
     launch_ops(c, chain, 1);
     for (int l = 0; l < md.n_layers; l++) {
         const int M = R / n_seq;
+        AttnParams ap;
+        ap.q = c->d_q_out; ap.ldq = d; ap.row_seq = c->d_row_seq; ap.row_pos = c->d_row_pos; ap.md = md;
+        ap.layer = l; ap.kc = (const bf*)c->kv_k; ap.vc = (const bf*)c->kv_v; ap.M = M;
+        ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
+        const bool plain = big && c->prompt_plain_bf16;
+        ap.out = c->d_attn_bf; ap.lo_row0 = plain ? -1 : rh; ap.debug_stale = c->attn_debug_stale;
+        ap.rows_per_block = 0;
+        ap.out_tile_rows = big && !plain ? rh : 0;
         if (M <= 32) {
-            AttnParams ap;
-            ap.q = c->d_q_out; ap.ldq = d; ap.row_seq = c->d_row_seq; ap.row_pos = c->d_row_pos; ap.md = md;
-            ap.layer = l; ap.kc = (const bf*)c->kv_k; ap.vc = (const bf*)c->kv_v; ap.M = M;
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             // Long contexts: the key loop (tensor-core work of 4 warps) outweighs everything that one CTA per
             // SM buys at short contexts, so the slices are doubled - two CTAs per SM, 8 warps on the keys.
             if (c->attn_long && ap.n_split * 2 <= 8) ap.n_split *= 2;
-            ap.part_o = c->d_attn_po; ap.part_ml = c->d_attn_pml; ap.counters = c->d_attn_cnt;
-            ap.out = c->d_attn_bf; ap.lo_row0 = rh; ap.debug_stale = c->attn_debug_stale;
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
             else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
-        } else if (md.dh == 128) {
-            LAUNCH(c, (k_attn_simple<bf, 128, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
         } else {
-            LAUNCH(c, (k_attn_simple<bf, 64, true>), dim3(md.H, R), 128, c->d_q_out, d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)c->d_attn_bf, rh);
+            // more than 32 rows: one sequence's prompt chunk (pass_forward_tokens, pass_prefill)
+            ap.debug_stale = 0;
+            if (md.dh == 128) { if (plain) launch_attn_chunk<128, false>(c, ap); else launch_attn_chunk<128, true>(c, ap); }
+            else              { if (plain) launch_attn_chunk<64, false>(c, ap); else launch_attn_chunk<64, true>(c, ap); }
         }
-        launch_ops(c, chain, build_layer_chain(c, R, npad, bm, l, head, chain));
+        launch_ops(c, chain, build_layer_chain(c, R, npad, bm, l, head, chain, big));
     }
     return PASS_OK;
 }
@@ -673,7 +728,8 @@ static void enqueue_step_any(pass_ctx* c, int k) {
     else enqueue_step<__nv_bfloat16>(c, k);
 }
 
-static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool want_logits) {
+// big: a prompt chunk of more than kMaxRows rows of a bf16 model on the tensor-core path (plain bf16 rows).
+static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool want_logits, bool big = false) {
     memcpy(c->pin_tok, tokens, sizeof(int) * n);
     CUDA_TRY(cudaMemcpyAsync(c->d_tok, c->pin_tok, sizeof(int) * n, cudaMemcpyHostToDevice, c->stream));
     if (c->md.dtype == PASS_DTYPE_FP32) {
@@ -686,7 +742,7 @@ static int run_tokens(pass_ctx* c, int seq, const int32_t* tokens, int n, bool w
                (const __nv_bfloat16*)c->la_emb, c->d_states, c->d_tok, seq, c->md.d, c->md.V, c->d_h,
                c->d_row_seq, c->d_row_pos);
         if (c->use_tc) {
-            const int rc = enqueue_layers_tc(c, n, 1, want_logits);
+            const int rc = enqueue_layers_tc(c, n, 1, want_logits, false, big);
             if (rc != PASS_OK) return rc;
         } else {
             enqueue_layers<__nv_bfloat16>(c, n);
@@ -797,7 +853,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     if (cudaMallocHost((void**)&c->pin_unif, sizeof(float) * cfg->max_batch * kUSlots) != cudaSuccess) return fail(PASS_ERR_CUDA);
     if (cudaMallocHost((void**)&c->pin_states, sizeof(SeqState) * cfg->max_batch) != cudaSuccess) return fail(PASS_ERR_CUDA);
     if (cudaMallocHost((void**)&c->pin_status, sizeof(int)) != cudaSuccess) return fail(PASS_ERR_CUDA);
-    if (cudaMallocHost((void**)&c->pin_tok, sizeof(int) * kMaxRows) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    if (cudaMallocHost((void**)&c->pin_tok, sizeof(int) * kRowsCap) != cudaSuccess) return fail(PASS_ERR_CUDA);
 
     // zero the small state region; rotary frequencies theta^(-2i/d_head) in float64
     if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
@@ -936,10 +992,19 @@ int pass_prefill(pass_ctx* c, int seq, const int32_t* tokens, int n) {
     }
     int rc = pass_reset(c, seq);
     if (rc != PASS_OK) return rc;
-    for (int s = 0; s < n - 1; s += kMaxRows) {
-        const int rows = std::min(kMaxRows, n - 1 - s);
-        rc = run_tokens(c, seq, tokens + s, rows, false);
+    // The prompt goes through the layers in chunks.  bf16 models on the tensor-core path: chunks of up to
+    // kRowsCap rows as large GEMMs over (feature tile, token tile) units with plain bf16 activations and causal
+    // flash attention, as long as more than kMaxRows rows remain; the last rows (and every other model) in
+    // chunks of up to kMaxRows rows through the step's own kernels.
+    const bool can_big = c->use_tc && getenv("PASS_NO_BIG_PREFILL") == nullptr;
+    for (int s = 0; s < n - 1;) {
+        const int left = n - 1 - s;
+        const bool big = can_big && left > kMaxRows;
+        const int big_rows = c->prompt_plain_bf16 ? kRowsCap : kRowsCap / 2;    // hi + lo parts take two buffer rows per token
+        const int rows = std::min(big ? big_rows : kMaxRows, left);
+        rc = run_tokens(c, seq, tokens + s, rows, false, big);
         if (rc != PASS_OK) return rc;
+        s += rows;
         LAUNCH(c, k_update_state, 1, 1, c->d_states, seq, 0, 0, rows, 0, 0, 0);
         CUDA_TRY(cudaStreamSynchronize(c->stream));   // pin_tok is reused by the next chunk
     }
@@ -1397,6 +1462,12 @@ int pass_linear_noalloc(pass_ctx* c, int which, int layer, const float* x_device
     if (rc == PASS_ERR_TIMEOUT)     // an abandoned launch may have left words in the shared slots
         CUDA_TRY(cudaMemset(scratch, 0xFF, kStaticPartialBytes));
     return rc;
+}
+
+int pass_set_prompt_precision(pass_ctx* c, int mode) {
+    if (!c || (mode != PASS_PROMPT_HI_LO && mode != PASS_PROMPT_BF16)) return PASS_ERR_INVALID_ARG;
+    c->prompt_plain_bf16 = mode == PASS_PROMPT_BF16;
+    return PASS_OK;
 }
 
 int pass_debug_set(pass_ctx* c, int hook, int value) {

@@ -10,7 +10,7 @@ namespace pass {
 
 constexpr int kMaxLA = PASS_MAX_LOOKAHEAD;          // 8
 constexpr int kMaxRows = PASS_MAX_ROWS;             // 128: rows of one step or one pass_forward_tokens call
-constexpr int kRowsCap = 256;                       // rows of one launch at most (prompt chunks): row tables, strides
+constexpr int kRowsCap = 2048;                      // rows of one launch at most (a prompt chunk): row tables, strides
 constexpr int kUSlots = 2 * kMaxLA + 1;             // uniforms per sequence and step
 constexpr int kVerifySplits = 8;                    // CTAs per logits row in the stats kernel
 constexpr int kVerifyThreads = 256;
