@@ -120,7 +120,7 @@ __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int r
                     if (sidx < p.n_split) v += vals[e][sidx] * sm_f[sidx * 32 + i];
                 const __nv_bfloat16 hi = __float2bfloat16_rn(v);
                 p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-                if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
             }
         }
     }
@@ -148,7 +148,9 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
 // MT = m-tiles of 16 rows per CTA (4 warps: MT = 4 gives every warp its own 16 rows and all keys of a block,
 // the usual flash-attention split for many rows).  HL = queries and probabilities as bf16 hi + lo pairs;
 // without it they are single bf16 values (prompt chunks in plain bf16, half the MMAs).
-template <int DH, int MT, bool CL, bool HL = true>
+// CHUNK = the rows are one sequence's prompt chunk (rows_per_block, out_tile_rows, optional lo parts); the
+// decode step's instances have it off and carry none of that code.
+template <int DH, int MT, bool CL, bool HL = true, bool CHUNK = false>
 __global__ void __maxnreg__(168)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
@@ -169,8 +171,8 @@ k_attn_fd(const AttnParams p) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int mt = warp % MT, part = warp / MT;
     // a decode step: rows b*M .. of sequence b; a prompt chunk: rows b*rows_per_block .. of the one sequence
-    const int row0 = p.rows_per_block ? b * p.rows_per_block : b * p.M;
-    const int M = p.rows_per_block ? min(p.rows_per_block, p.M - row0) : p.M;
+    const int row0 = CHUNK ? b * p.rows_per_block : b * p.M;
+    const int M = CHUNK ? min(p.rows_per_block, p.M - row0) : p.M;
     // one thread reads the tables for all, so that the whole CTA works from the same pair even if it
     // reads while they are being written
     __shared__ int s_tab[2];
@@ -198,7 +200,7 @@ k_attn_fd(const AttnParams p) {
     slice(s_tab[0], max(0, s_tab[1] - p.debug_stale));
     // rows of this launch's own chunk ahead of this block are cache rows the awaited kernel writes: in chunk
     // mode only positions before the chunk's first row may be fetched early
-    const int early_len = p.rows_per_block ? min(len, *(volatile const int*)(p.row_pos)) : len;
+    const int early_len = CHUNK ? min(len, *(volatile const int*)(p.row_pos)) : len;
     const uint32_t sK = smem_u32(smem_attn), sV = sK + kAttnStages * TILE_BYTES;
 
     auto load_block = [&](int blk) {
@@ -423,9 +425,9 @@ k_attn_fd(const AttnParams p) {
             const float v = acc / ll;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
             const int g_row = row0 + i;
-            const int o_row = p.out_tile_rows ? (g_row / p.out_tile_rows) * 2 * p.out_tile_rows + g_row % p.out_tile_rows : g_row;
+            const int o_row = (CHUNK && p.out_tile_rows) ? (g_row / p.out_tile_rows) * 2 * p.out_tile_rows + g_row % p.out_tile_rows : g_row;
             p.out[(size_t)o_row * p.md.d + head * DH + dcol] = hi;
-            if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + o_row) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            if (!CHUNK || p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + o_row) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
         } else if (CL) {
             float* cl_o = sm_o + 4 * 16 * DH + 128;          // [32][DH], behind the warp staging area
             float* cl_ml = cl_o + 32 * DH;                   // [32][2]
@@ -468,7 +470,7 @@ k_attn_fd(const AttnParams p) {
             const int dcol = idx % DH;
             const __nv_bfloat16 hi = __float2bfloat16_rn(v);
             p.out[(size_t)(row0 + i) * p.md.d + head * DH + dcol] = hi;
-            if (p.lo_row0 >= 0) p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            p.out[(size_t)(p.lo_row0 + row0 + i) * p.md.d + head * DH + dcol] = __float2bfloat16_rn(v - __bfloat162float(hi));
         }
         cluster_sync_all();                                  // nobody leaves while its memory is still being read
         return;

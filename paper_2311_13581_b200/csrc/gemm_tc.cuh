@@ -318,17 +318,21 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 // loaded (so that this trip to L2 overlaps with another); nullptr = load them here.
 // g_pre / cs_pre: likewise the next norm's gain for this feature (kEpiResid) and the eight rotation pairs
 // (kEpiQKV), fetched by the caller while it was still waiting for the accumulator.
-template <int NR>
+template <int NR, bool BIG>
 __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[NR],
                                           const float* hv_pre = nullptr, const float* g_pre = nullptr,
                                           const float2* cs_pre = nullptr) {
     const int L = ec.lane_in_tile;
+    // the step's kernel (BIG = false) has one token tile of hi | lo rows: these fold to constants there
+    const int row_base = BIG ? ec.row_base : 0, out_row_base = BIG ? ec.out_row_base : 0;
+    const int rows_live = BIG ? ec.rows_live : p.R;
+    const bool has_lo = BIG ? p.has_lo != 0 : true;
     if (p.epi == kEpiLogits) {
         const int n = tile * kTileN + L;
         if (n < p.n_out) {
 #pragma unroll
             for (int j = 0; j < NR; j++)
-                if (c0 + j < ec.rows_live) p.logits[(size_t)(ec.row_base + c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
+                if (c0 + j < rows_live) p.logits[(size_t)(row_base + c0 + j) * p.n_out + n] = v[j] * ec.s_rstd[c0 + j];
         }
     } else if (p.epi == kEpiQKV) {
         const int d = p.md.d, dh = p.md.dh;
@@ -340,21 +344,21 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         const size_t head_off = ((size_t)head * p.md.cap) * dh + i;
 #pragma unroll
         for (int j = 0; j < NR; j++) {
-            const int r = min(c0 + j, ec.rows_live - 1);
+            const int r = min(c0 + j, rows_live - 1);
             kvo[j] = (size_t)ec.s_kvoff[r] + head_off;
-            cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)(ec.row_base + r) * (dh / 2) + (i >> 1));
+            cs[j] = cs_pre ? cs_pre[j] : __ldg(p.rope_cs + (size_t)(row_base + r) * (dh / 2) + (i >> 1));
         }
 #pragma unroll
         for (int j = 0; j < NR; j++) {
             const int r = c0 + j;
-            const float x = v[j] * (r < ec.rows_live ? ec.s_rstd[r] : 0.f);
+            const float x = v[j] * (r < rows_live ? ec.s_rstd[r] : 0.f);
             const float other = __shfl_xor_sync(0xffffffffu, x, 1);
-            if (r < ec.rows_live) {
+            if (r < rows_live) {
                 if (which == 2) {
                     p.vc[kvo[j]] = __float2bfloat16_rn(x);
                 } else {
                     const float y = (i & 1) ? other * cs[j].y + x * cs[j].x : x * cs[j].x - other * cs[j].y;
-                    if (which == 0) p.q_out[(size_t)(ec.row_base + r) * d + c] = y;
+                    if (which == 0) p.q_out[(size_t)(row_base + r) * d + c] = y;
                     else p.kc[kvo[j]] = __float2bfloat16_rn(y);
                 }
             }
@@ -367,19 +371,19 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         float ss[NR], hv[NR];
 #pragma unroll
         for (int j = 0; j < NR; j++)      // all loads first: they are independent of the stores below
-            hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < ec.rows_live && n < d) ? __ldcg(p.h + (size_t)(ec.row_base + c0 + j) * d + n) : 0.f);
+            hv[j] = hv_pre ? hv_pre[j] : ((c0 + j < rows_live && n < d) ? __ldcg(p.h + (size_t)(row_base + c0 + j) * d + n) : 0.f);
 #pragma unroll
         for (int j = 0; j < NR; j++) {
-            const int r = ec.row_base + c0 + j;
+            const int r = row_base + c0 + j;
             float hn = 0.f;
-            if (c0 + j < ec.rows_live && n < d) {
+            if (c0 + j < rows_live && n < d) {
                 hn = hv[j] + v[j];
                 p.h[(size_t)r * d + n] = hn;
                 __nv_bfloat16 hi, lo;
                 split_bf16(hn * g, hi, lo);
-                const size_t orow = (size_t)(ec.out_row_base + c0 + j);
+                const size_t orow = (size_t)(out_row_base + c0 + j);
                 p.xn_out[orow * d + n] = hi;
-                if (p.has_lo) p.xn_out[(orow + p.xn_lo_row0) * d + n] = lo;
+                if (has_lo) p.xn_out[(orow + p.xn_lo_row0) * d + n] = lo;
             }
             ss[j] = hn * hn;
         }
@@ -396,8 +400,8 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
             for (int j = 0; j < NR; j++) ec.s_x[warp_q * NR + j] = ss[j];
         }
         epi_bar();
-        if (L < NR && c0 + L < ec.rows_live)
-            p.sumsq_out[(size_t)tile * kRowsCap + ec.row_base + c0 + L] =
+        if (L < NR && c0 + L < rows_live)
+            p.sumsq_out[(size_t)tile * kRowsCap + row_base + c0 + L] =
                 ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
     } else {  // kEpiSwiGLU: lanes 0..63 gate features 64*tile + L, lanes 64..127 the matching up features
         // Both halves of the threads work after the exchange: a gate lane finishes the even rows of its
@@ -411,15 +415,15 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         if (n < p.n_out) {
 #pragma unroll
             for (int j = 0; j < NR; j++) {
-                if (c0 + j < ec.rows_live && ((j & 1) == (L >> 6))) {
+                if (c0 + j < rows_live && ((j & 1) == (L >> 6))) {
                     const float rs = ec.s_rstd[c0 + j];
                     const float mine = v[j] * rs, theirs = ec.s_x[other * 9 + j] * rs;
                     const float g = L < 64 ? mine : theirs, u = L < 64 ? theirs : mine;
                     __nv_bfloat16 hi, lo;
                     split_bf16(g / (1.f + __expf(-g)) * u, hi, lo);
-                    const size_t orow = (size_t)(ec.out_row_base + c0 + j);
+                    const size_t orow = (size_t)(out_row_base + c0 + j);
                     p.act_out[orow * p.n_out + n] = hi;
-                    if (p.has_lo) p.act_out[(orow + p.xn_lo_row0) * p.n_out + n] = lo;
+                    if (has_lo) p.act_out[(orow + p.xn_lo_row0) * p.n_out + n] = lo;
                 }
             }
         }
@@ -579,8 +583,10 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
     __shared__ int s_epi_done;
     __shared__ int s_last;
     __shared__ int s_epi_fail;
-    __shared__ float s_rstd[kTokTile];
-    __shared__ unsigned long long s_kvoff[kTokTile];
+    // (the step's kernel shares its SM with an attention CTA of 96 KB: every byte of static shared memory counts,
+    // 512 bytes more and the two no longer fit side by side)
+    __shared__ float s_rstd[BIG ? kTokTile : kMaxRows];
+    __shared__ unsigned long long s_kvoff[BIG ? kTokTile : kMaxRows];
     __shared__ float s_x[128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
@@ -901,7 +907,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                             if (!whole)
                                 ll_gather(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
                             if (et == 0 && c0 == 0 && !whole) PASS_TRACE(oi, 5);
-                            epi_store<kLLRows>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
+                            epi_store<kLLRows, BIG>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
                                                p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs9 : nullptr);
                         }
                         if (!whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
@@ -935,7 +941,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         for (int j = 0; j < 8; j++) hi[j] += lo[j];
                     }
                     if (whole) {
-                        epi_store<8>(p, ec, ftile, c0, hi, ahead ? hv_cur : nullptr, ahead ? &g_res : nullptr);
+                        epi_store<8, BIG>(p, ec, ftile, c0, hi, ahead ? hv_cur : nullptr, ahead ? &g_res : nullptr);
                         if (ahead) {
 #pragma unroll
                             for (int j = 0; j < 8; j++) hv_cur[j] = hv_nxt[j];
@@ -1001,7 +1007,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                                     }
                                 }
                             }
-                            epi_store<8>(p, ec, pc.tile, c0, acc);
+                            epi_store<8, BIG>(p, ec, pc.tile, c0, acc);
                         }
                     }
                 }

@@ -599,7 +599,7 @@ static void launch_attn_chunk(pass_ctx* c, AttnParams ap) {
     constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
     bool& set = c->attn_attr_set[DH * 8 + 4 * 2 + (HL ? 64 : 32)];
     if (!set) {
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, 4, false, HL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, 4, false, HL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
         set = true;
     }
     cudaLaunchConfig_t cfg;
@@ -613,7 +613,7 @@ static void launch_attn_chunk(pass_ctx* c, AttnParams ap) {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = c->use_pdl ? 1 : 0;
-    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, 4, false, HL>, ap), "k_attn_fd (chunk) launch");
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, 4, false, HL, true>, ap), "k_attn_fd (chunk) launch");
     c->launches++;
 }
 
