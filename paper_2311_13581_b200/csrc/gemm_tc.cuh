@@ -51,7 +51,6 @@ enum GemmEpilogue { kEpiLogits = 0, kEpiQKV = 1, kEpiResid = 2, kEpiSwiGLU = 3 }
 
 struct GemmParams {
     int n_tiles, kb_per_tile;
-    int K;                         // elements of an activation row (the GEMM's inner dimension)
     int seg_tiles0, seg_tiles1;    // plain mode: tiles of weight map 0 and 1 (the rest is map 2)
     int interleave;                // 1: tile t = rows [64t, 64t+64) of map 0 (gate) and of map 1 (up)
     int packed;                    // 1: the weight maps are over the packed copy [tile][k-block][box rows][64]
@@ -520,13 +519,6 @@ struct ChainParams {
     int op_target[kMaxOps];    // value of op_done[i] once this launch's GEMM i is complete
     int* status;
     unsigned long long* trace;     // optional %globaltimer stamps [kMaxOps][CTA][8] of this launch (nullptr = off)
-    // Activations handed from GEMM j-1 to GEMM j of the launch as data that is its own flag (9..16 token rows,
-    // see poll_tile): bit j of poll_mask = GEMM j takes its first activation tiles from poll_src[j] by polling.
-    int poll_mask;
-    const __nv_bfloat16* poll_src[kMaxOps];     // [32][K]: hi rows 0.., lo rows 16..; EMPTY (all bits set) until written
-    int reset_n;                                // buffers of that kind which this launch marks EMPTY again at its start
-    __nv_bfloat16* reset_buf[6];                // (the ones the launch before the previous one filled; see the host side)
-    int reset_K[6];
     GemmParams op[kMaxOps];
 };
 // Only every 16th CTA leaves stamps: reads of %globaltimer from all CTAs at once queue up behind one another
@@ -547,75 +539,6 @@ __device__ __forceinline__ bool wait_count(const int* counter, int target, volat
         }
         __nanosleep(64);
     }
-}
-
-// ------------------------------------------------------------------------------------ polled activation tiles
-// Between two GEMMs of a launch the activations (9..16 token rows as bf16 hi + lo rows) can be handed over as
-// data that is its own flag.  A buffer element is EMPTY (0xffff, a NaN pattern the conversion from float never
-// makes) until the finishing epilogue of the previous GEMM stores it; the consumer's loader warp copies the
-// rows of a tile into the shared-memory stage with 16-byte asynchronous copies, looks at what arrived and
-// fetches again whatever still holds an EMPTY element.  Against counter + TMA this takes the release fence, the
-// flag's round trip and the TMA's latency out of the hand-over: the data is in shared memory one trip to L2
-// after it was stored.  Once the previous GEMM's completion counter has been seen the remaining tiles of the
-// GEMM are fetched by TMA as before.  Each launch uses the buffers of its parity and re-empties the other
-// parity's (filled two launches ago, read by the launch before this one, which has completed).
-__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// phase complete?  Unlike try_wait this never parks the thread.
-__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-__device__ __forceinline__ void g_cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void g_cp_async_commit_wait() {
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts128_zero(uint32_t addr) {
-    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
-}
-// One lane's share of a [2 R rows x 64 columns] activation tile (k-block kb): chunk q = 16 bytes, rows 0..R-1
-// are the hi rows, R..2R-1 the lo rows (buffer rows 16..).  CHECK = false: request the chunks.  CHECK = true: look
-// at them in shared memory and request again those that are not complete; returns true when this lane's all are.
-template <bool CHECK>
-__device__ __forceinline__ bool poll_tile(uint32_t b_tile, const __nv_bfloat16* src, int K, int R, int kb, int lane) {
-    bool complete = true;
-    for (int q = lane; q < 16 * R; q += 32) {
-        const int rr = q >> 3, c = q & 7;
-        const int row = rr < R ? rr : 16 + rr - R;
-        const int col = kb * kBlockK + c * 8;
-        const uint32_t dst = b_tile + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4));
-        if (col >= K) {                       // beyond the matrix (ragged last k-block): zeros, as TMA would fill
-            if (!CHECK) sts128_zero(dst);
-            continue;
-        }
-        const __nv_bfloat16* g = src + (size_t)row * K + col;
-        if (!CHECK) {
-            g_cp_async16(dst, g);
-        } else {
-            const uint4 w = lds128(dst);
-            const uint32_t any = __vcmpeq2(w.x, 0xffffffffu) | __vcmpeq2(w.y, 0xffffffffu) |
-                                 __vcmpeq2(w.z, 0xffffffffu) | __vcmpeq2(w.w, 0xffffffffu);
-            if (any) {
-                complete = false;
-                g_cp_async16(dst, g);
-            }
-        }
-    }
-    return complete;
 }
 
 // weight tile of (tile, k-block): box index 0/1 -> (map, row); plain mode has a single 128-row box.
@@ -758,113 +681,27 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
         }
     } else if (warp == 6) {
         // ---------------------------------------------------------------- activation producer
-        // Lane 0 issues the TMA requests; the whole warp takes part only while a GEMM's first tiles are polled.
-        const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-        int fill = 0;
-        bool ok = true;
-        Piece pc;
-        if (lane == 0) griddep_wait();         // the first GEMM's activations are the previous kernel's output
-        __syncwarp();
-        for (int oi = 0; ok && oi < cp.n_ops; oi++) {
-            const GemmParams& p = cp.op[oi];
-            const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
-            const bool polled = !BIG && ((cp.poll_mask >> oi) & 1);
-            int it = 0, kb = 0;
-            bool have = fetch_piece(oi, 0, pc);
-            if (have) kb = pc.kb0;
-            if (polled) {
-                // A window of up to NB stages whose tiles have been requested and are looked at round after round
-                // (one trip to L2 per round for all of them); a stage leaves the window when its tile is complete.
-                constexpr int NB = 6;
-                const __nv_bfloat16* src = cp.poll_src[oi];
-                const long long t_op = clock64();
-                int ws[NB], wkb[NB];
-                uint32_t pend = 0;             // bit j: window slot j holds a stage whose tile is not complete yet
-                bool done = false, stamped = false;
-                while (ok && !done && (have || pend)) {
-                    bool progressed = false;
-                    while (have && pend != (1u << NB) - 1) {          // admit stages that are free right now
-                        const int s = fill % S;
-                        int fr = 0;
-                        if (lane == 0) fr = (int)mbar_test_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1);
-                        if (!__shfl_sync(0xffffffffu, fr, 0)) break;
-                        const uint32_t dst = tiles_base + s * stage_bytes;
-                        if (lane == 0 && p.interleave) {       // the stage's second weight box is this role's job
-                            const CUtensorMap* m;
-                            int y, wx, wy;
-                            weight_box(p, maps.m[oi], pc.tile, 1, m, y);
-                            weight_xy(p, y, kb, wx, wy);
-                            mbar_expect_tx_only(bar_full + 8 * s, kATileBytes / 2);
-                            tma_load_2d(dst + kATileBytes / 2, m, bar_full + 8 * s, wx, wy, pol_w);
-                        }
-                        poll_tile<false>(dst + kATileBytes, src, p.K, p.R, kb, lane);
-                        bool placed = false;
-#pragma unroll
-                        for (int j = 0; j < NB; j++)
-                            if (!placed && !((pend >> j) & 1u)) { ws[j] = s; wkb[j] = kb; pend |= 1u << j; placed = true; }
-                        fill++;
-                        progressed = true;
-                        if (++kb >= pc.kb1) {
-                            it++;
-                            have = fetch_piece(oi, it, pc);
-                            if (have) kb = pc.kb0;
-                        }
-                    }
-                    g_cp_async_commit_wait();
-#pragma unroll
-                    for (int j = 0; j < NB; j++) {
-                        if (!((pend >> j) & 1u)) continue;
-                        const bool mine = poll_tile<true>(tiles_base + ws[j] * stage_bytes + kATileBytes, src, p.K, p.R, wkb[j], lane);
-                        if (!__all_sync(0xffffffffu, mine)) continue;
-                        fence_proxy_async();       // this lane's copies into shared memory before the tensor core reads them
-                        __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(bar_full + 8 * ws[j]);
-                            if (!stamped) PASS_TRACE(oi, 0);
-                        }
-                        stamped = true;
-                        pend &= ~(1u << j);
-                        progressed = true;
-                    }
-                    g_cp_async_commit_wait();              // what was requested again (nothing stays in flight)
-                    if (lane == 0) *(volatile int*)&s_issued_b = fill - __popc(pend);
-                    if (pend == 0) {
-                        // the previous GEMM complete?  Then every element is there and TMA fetches the rest.
-                        int d = 0;
-                        if (lane == 0) {
-                            int v;
-                            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(cp.op_done + oi - 1) : "memory");
-                            d = v >= cp.op_target[oi - 1];
-                        }
-                        done = __shfl_sync(0xffffffffu, d, 0) != 0;
-                    }
-                    if (!progressed) {
-                        const bool giveup = *(volatile int*)&s_abort || clock64() - t_op > kWaitCycles;
-                        if (__any_sync(0xffffffffu, giveup)) {
-                            if (lane == 0) { s_abort = 1; atomicOr(cp.status, kStatusTimeout); }
-                            ok = false;
-                        }
-                        __nanosleep(100);
-                    }
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+            int fill = 0;
+            bool ok = true;
+            Piece pc;
+            griddep_wait();                    // the first GEMM's activations are the previous kernel's output
+            for (int oi = 0; ok && oi < cp.n_ops; oi++) {
+                const GemmParams& p = cp.op[oi];
+                const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
+                if (oi > 0) {
+                    // activations of this GEMM = results of the previous one, written by other SMs
+                    if (!wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status)) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
                 }
-                if (lane == 0 && ok && have) asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
-            } else if (oi > 0) {
-                // activations of this GEMM = results of the previous one, written by other SMs
-                int w = 1;
-                if (lane == 0) {
-                    w = wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status) ? 1 : 0;
-                    if (w) asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy data -> TMA reads
-                }
-                if (!__shfl_sync(0xffffffffu, w, 0)) { ok = false; break; }
-            }
-            if (lane == 0 && ok) {
-                if (!polled) PASS_TRACE(oi, 0);
-                for (; ok && have; it++, have = fetch_piece(oi, it, pc), kb = have ? pc.kb0 : 0) {
+                PASS_TRACE(oi, 0);
+                for (int it = 0; ok && fetch_piece(oi, it, pc); it++) {
                     const CUtensorMap* m;
                     int y;
                     weight_box(p, maps.m[oi], (BIG && p.n_tok_tiles > 0) ? pc.tile / p.n_tok_tiles : pc.tile, 1, m, y);
                     const int b_row0 = (BIG && p.n_tok_tiles > 0) ? (pc.tile % p.n_tok_tiles) * p.npad : 0;    // token tile
-                    for (; kb < pc.kb1; kb++) {
+                    for (int kb = pc.kb0; kb < pc.kb1; kb++) {
                         const int s = fill % S;
                         if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
                         const uint32_t dst = tiles_base + s * stage_bytes;
@@ -882,9 +719,6 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     }
                 }
             }
-            // every lane goes on from where lane 0 stopped
-            fill = __shfl_sync(0xffffffffu, fill, 0);
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issue
@@ -929,19 +763,6 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
         ec.s_kvoff = s_kvoff;
         const int et = (warp - 2) * 32 + lane;        // 0..127
         griddep_wait();
-        if (!BIG && cp.reset_n > 0) {
-            // polled activation buffers of the other parity: every launch that could read them has completed
-            const int Rr = cp.op[0].R;
-            for (int b = 0; b < cp.reset_n; b++) {
-                uint4* base = reinterpret_cast<uint4*>(cp.reset_buf[b]);
-                const int K8 = cp.reset_K[b] / 8, total = 2 * Rr * K8;
-                for (int q = cta * 128 + et; q < total; q += G * 128) {
-                    const int rr = q / K8, c8 = q % K8;
-                    const int row = rr < Rr ? rr : 16 + rr - Rr;
-                    base[(size_t)row * K8 + c8] = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
-                }
-            }
-        }
         int pidx = 0;
         bool ok = true;
         Piece pc;

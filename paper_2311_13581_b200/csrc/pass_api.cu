@@ -37,7 +37,6 @@ struct Layout {
     size_t ll_ws;
     size_t attn_po, attn_pml, attn_cnt, chain_flags;
     size_t packed, packed_bytes;       // the weights in streaming order (see k_pack_weight)
-    size_t poll, poll_bytes;           // polled activation buffers: 2 parities x {[32][d], [32][f], [32][d]} bf16
     size_t total;
 };
 
@@ -98,7 +97,6 @@ Layout make_layout(const pass_config& c) {
     L.xn_bf = L.attn_bf = L.act_bf = L.q_out = L.sumsq_a = L.sumsq_b = L.partial_ws = L.counters = 0;
     L.attn_po = L.attn_pml = L.attn_cnt = L.chain_flags = 0;
     L.packed = L.packed_bytes = 0;
-    L.poll = L.poll_bytes = 0;
     if (c.dtype == PASS_DTYPE_BF16) {
         L.xn_bf = cv.take(RC * d * 2);           // kRowsCap plain rows, or hi rows + lo rows of a step
         L.attn_bf = cv.take(RC * d * 2);
@@ -114,8 +112,6 @@ Layout make_layout(const pass_config& c) {
         L.attn_pml = cv.take(slices * 32 * 2 * 4);
         L.attn_cnt = cv.take(B * c.n_heads * 4);
         L.chain_flags = cv.take(2 * kMaxOps * 4);
-        L.poll_bytes = 2 * (2 * 32 * d + 32 * f) * 2;
-        L.poll = cv.take(L.poll_bytes);
         L.packed_bytes = (size_t)c.n_layers * (4 * packed_matrix_bytes(d, d, 128) + 2 * packed_matrix_bytes(f, d, 64) +
                                                packed_matrix_bytes(d, f, 128)) + packed_matrix_bytes(V, d, 128);
         L.packed = cv.take(L.packed_bytes);
@@ -166,13 +162,6 @@ struct pass_ctx {
     std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
     bool use_tc = false;
-    // Polled hand-over of activations between the GEMMs of a launch (9..16 token rows, see poll_tile): buffers
-    // [parity][0: O-proj -> gate|up, 1: gate|up -> down, 2: down -> QKV / head], their tensor maps (box of 32 rows),
-    // and the number of chain launches since the forward began (its parity picks the buffers).
-    bool use_poll = false;             // PASS_POLL=1
-    __nv_bfloat16* d_poll[2][3] = {{nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr}};
-    CUtensorMap tm_poll[2][3];
-    int chain_parity = 0;
     bool prompt_plain_bf16 = false;    // pass_set_prompt_precision: long prompts with plain bf16 activations
     bool packed = false;               // the GEMMs stream the packed copy of the weights (PASS_NO_PACK: the caller's matrices)
     char* d_packed = nullptr;
@@ -347,7 +336,6 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.n_tiles = n_tiles;
-    p.K = K;
     p.kb_per_tile = (K + kBlockK - 1) / kBlockK;
     p.seg_tiles0 = p.seg_tiles1 = 1 << 30;
     p.npad = npad;
@@ -372,8 +360,6 @@ static GemmParams gemm_base(pass_ctx* c, int R, int npad, int K, int n_tiles, in
 struct ChainOp {
     GemmParams p;
     CUtensorMap a0, a1, a2, b;
-    const __nv_bfloat16* poll_src = nullptr;   // the activations come from this polled buffer (if an earlier GEMM of the launch fills it)
-    int reset_mask = 0;                        // first entry of a launch: parities whose polled buffers the launch re-empties
 };
 
 // The tail of the verify scratch (E, [kMaxRows][V] doubles) doubles as the trace buffer: its rows beyond the
@@ -405,14 +391,6 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
         cp.op_target[j] = c->chain_done_total[j];
     }
     cp.status = c->d_status;
-    for (int j = 1; j < n_ops; j++)
-        if (ops[j].poll_src) { cp.poll_mask |= 1 << j; cp.poll_src[j] = ops[j].poll_src; }
-    for (int par = 0; par < 2; par++)
-        if ((ops[0].reset_mask >> par) & 1)
-            for (int q = 0; q < 3; q++) {
-                cp.reset_buf[cp.reset_n] = c->d_poll[par][q];
-                cp.reset_K[cp.reset_n++] = q == 1 ? c->md.f : c->md.d;
-            }
     if (c->trace && c->trace_launch < kTraceLaunches && trace_base(c))
         cp.trace = trace_base(c) + (size_t)(c->trace_launch++) * kMaxOps * kMaxCtas * 8;
     const size_t region = (size_t)kMaxCtas * 2 * kMaxRows * kTileN;      // floats per GEMM of the chain
@@ -570,7 +548,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
     const ModelDims& md = c->md;
     const int d = md.d, f = md.f, dt = d / kTileN;
     int n = 0;
-    for (int j = 0; j < kMaxOps; j++) { ch[j].poll_src = nullptr; ch[j].reset_mask = 0; }
     {   // attention output projection + residual; prepares the input of the feed-forward norm
         ChainOp& o = ch[n++];
         o.p = gemm_base(c, R, npad, d, dt, d, kEpiResid);
@@ -605,19 +582,6 @@ static int build_layer_chain(pass_ctx* c, int R, int npad, const pass_ctx::BMaps
         o.p.logits = c->d_logits;
         o.a0 = o.a1 = o.a2 = c->tm_lm; o.b = bm->xn;
         if (big) set_big(c, o.p, R, (md.V + kTileN - 1) / kTileN);
-    }
-    if (!big && npad == 32 && c->use_poll) {
-        // 9..16 token rows: the activations travel between the GEMMs of this launch through the polled buffers
-        // of the launch's parity; the launch re-empties the other parity's
-        const int par = c->chain_parity & 1;
-        c->chain_parity++;
-        ch[0].p.xn_out = c->d_poll[par][0];
-        ch[1].b = c->tm_poll[par][0]; ch[1].poll_src = c->d_poll[par][0];
-        ch[1].p.act_out = c->d_poll[par][1];
-        ch[2].b = c->tm_poll[par][1]; ch[2].poll_src = c->d_poll[par][1];
-        ch[2].p.xn_out = c->d_poll[par][2];
-        if (n > 3) { ch[3].b = c->tm_poll[par][2]; ch[3].poll_src = c->d_poll[par][2]; }
-        ch[0].reset_mask = 1 << (par ^ 1);
     }
     return n;
 }
@@ -673,8 +637,6 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
     // Kernels of a step: QKV_0 | per layer: attention, then ONE launch running
     // O-projection -> gate|up -> down -> (next layer's QKV, or the output head after the last layer).
     chain[0] = op_qkv(c, R, npad, bm, 0, big);
-    c->chain_parity = 0;
-    if (!big && npad == 32 && c->use_poll) chain[0].reset_mask = 3;     // a forward starts with every polled buffer EMPTY
     launch_ops(c, chain, 1);
     for (int l = 0; l < md.n_layers; l++) {
         const int M = R / n_seq;
@@ -870,16 +832,6 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->d_attn_pml = (float*)(w + L.attn_pml);
         c->d_attn_cnt = (int*)(w + L.attn_cnt);
         c->d_chain_flags = (int*)(w + L.chain_flags);
-        {
-            __nv_bfloat16* pb = (__nv_bfloat16*)(w + L.poll);
-            const size_t d = cfg->d_model, f = cfg->d_ffn;
-            for (int par = 0; par < 2; par++) {
-                c->d_poll[par][0] = pb; pb += 32 * d;
-                c->d_poll[par][1] = pb; pb += 32 * f;
-                c->d_poll[par][2] = pb; pb += 32 * d;
-            }
-            c->use_poll = getenv("PASS_POLL") != nullptr && getenv("PASS_NO_CHAIN") == nullptr;
-        }
         c->d_packed = w + L.packed;
         c->packed = getenv("PASS_NO_PACK") == nullptr;
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
@@ -910,13 +862,6 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     // the hand-over slots of the <=16-row GEMMs are EMPTY (all bits set) whenever no launch is using them
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.ll_ws, 0xFF, kLLRegionBytes * kMaxOps, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
-    // so are the polled activation buffers
-    if (cfg->dtype == PASS_DTYPE_BF16) {
-        if (cudaMemsetAsync(w + L.poll, 0xFF, L.poll_bytes, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
-        for (int par = 0; par < 2; par++)
-            for (int q = 0; q < 3; q++)
-                if (!make_map(&c->tm_poll[par][q], c->d_poll[par][q], 32, q == 1 ? cfg->d_ffn : cfg->d_model, 32)) return fail(PASS_ERR_CUDA);
-    }
     std::vector<double> inv(cfg->d_head / 2);
     for (int i = 0; i < cfg->d_head / 2; i++)
         inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
@@ -1076,7 +1021,6 @@ int pass_prefill(pass_ctx* c, int seq, const int32_t* tokens, int n) {
 // it goes back to the idle state, in stream order, before the next launch.
 static cudaError_t scrub_after_timeout(pass_ctx* c) {
     cudaError_t e = cudaMemsetAsync(c->d_ll, 0xFF, kLLRegionBytes * kMaxOps, c->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->L.poll, 0xFF, c->L.poll_bytes, c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->d_counters, 0, 4096 * sizeof(int), c->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(c->d_attn_cnt, 0, (size_t)c->md.B * c->md.H * sizeof(int), c->stream);
     return e;
@@ -1419,8 +1363,6 @@ int pass_debug_time_linear(pass_ctx* c, int which, int R, int n_launches, float*
     };
     if (which == 9) {              // rows at position 0 of sequence 0: the QKV epilogue needs valid row tables
         chain_counters_clear(c);
-        c->chain_parity = 0;
-        CUDA_TRY(cudaMemsetAsync(c->ws + c->L.poll, 0xFF, c->L.poll_bytes, c->stream));
         CUDA_TRY(cudaMemsetAsync(c->d_row_seq, 0, sizeof(int) * kMaxRows, c->stream));
         CUDA_TRY(cudaMemsetAsync(c->d_row_pos, 0, sizeof(int) * kMaxRows, c->stream));
     }
