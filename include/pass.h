@@ -202,6 +202,55 @@ int pass_forward_tokens(pass_ctx *ctx, int seq, const int32_t *tokens, int n,
 #define PASS_PROMPT_BF16  1
 int pass_set_prompt_precision(pass_ctx *ctx, int mode);
 
+/*
+ * Training of the look-ahead embeddings (Supplementary material, "Training details"; section "Look-ahead
+ * embeddings").  The model stays frozen; the only parameters are the first L rows of the look-ahead table.
+ * For a training sequence w_0 .. w_{S-1} and a position n the model reads (w_0 .. w_n, LA_1 .. LA_L) in one
+ * causal pass; the output at LA_t is the draft of the token t + 1 places after w_n (Algorithm 1, drafting
+ * phase), so the loss of the sequence is the mean over t = 1..L of the cross entropy of that output against
+ * w_{n+1+t}; a batch averages over its sequences.  The gradient is taken with respect to the L look-ahead input
+ * rows only (because of the causal mask no other row depends on them, so the backward pass runs over those rows
+ * alone) and applied with AdamW (decoupled weight decay) under a linear warm-up followed by half a cosine down to
+ * zero; the paper gives lr 0.01, 2000 warm-up steps, 10000 steps, batches of 8 sequences, and names no other
+ * hyper-parameter (betas, eps and weight decay are the caller's; 0.9 / 0.999 / 1e-8 / 0.01 are customary).
+ * bf16 models on the tensor-core path only.  float32 master rows, moments and everything the two passes keep live
+ * in a training workspace of the caller's (pass_train_workspace_bytes: dominated by a transposed copy of the
+ * weights in streaming order, as large as the weights).
+ */
+typedef struct {
+    float lr, beta1, beta2, eps, weight_decay;
+    int warmup_steps, total_steps;
+} pass_train_config;
+
+/* Bytes of the training workspace for L look-ahead rows and batches of up to max_seqs sequences
+ * (L <= k_max, max_seqs <= max_batch, L * max_seqs <= PASS_MAX_ROWS); 0 on a bad argument or a float32 config. */
+size_t pass_train_workspace_bytes(const pass_config *cfg, int L, int max_seqs);
+/* Set up training: builds the transposed weight copies, copies rows 0..k_max-1 of the context's look-ahead table
+ * into float32 master rows, clears the moments and the step count.  train_ws_device: caller-allocated device
+ * memory, 256-byte aligned, borrowed until pass_destroy or the next pass_train_init.  Synchronises.
+ * Errors: INVALID_ARG, CAPACITY (workspace too small), STATE (weights not loaded, float32 model), CUDA. */
+int pass_train_init(pass_ctx *ctx, void *train_ws_device, size_t bytes, const pass_train_config *hp, int L,
+                    int max_seqs);
+/*
+ * One training step on n_seqs sequences (sequence b uses cache slot b, whose contents are replaced).
+ *   tokens    : HOST [n_seqs][stride] token ids; of sequence b the entries 0 .. positions[b] + 1 + L are read.
+ *   positions : HOST [n_seqs], the index n of the last prompt token of each sequence (n >= 0, n + 1 + L < stride,
+ *               n + 1 + L <= kv_capacity).
+ *   apply_update : 1 = AdamW update of the master rows and step count + 1; 0 = loss and gradient only.
+ *   loss_out  : HOST float, the batch loss (before the update).
+ * Runs the prompt parts through pass_prefill's path, then forward and backward over the n_seqs * L look-ahead
+ * rows.  Synchronises.  Errors: INVALID_ARG, CAPACITY, STATE (pass_train_init not called), TIMEOUT, CUDA.
+ */
+int pass_train_step(pass_ctx *ctx, const int32_t *tokens, int stride, const int32_t *positions, int n_seqs,
+                    int apply_update, float *loss_out);
+/* Read back [L][d_model] float32 rows to HOST memory: the master rows or the gradient of the last step. */
+#define PASS_TRAIN_LA    0
+#define PASS_TRAIN_GRAD  1
+int pass_train_get(pass_ctx *ctx, int what, float *dst_host, size_t bytes);
+/* Write the trained rows, rounded to bf16, into rows 0..L-1 of a look-ahead table on the DEVICE (for example the
+ * one given to pass_load_weights, which later steps then read). */
+int pass_train_export(pass_ctx *ctx, void *la_emb_device);
+
 /* Forget everything about sequence `seq` (len = 0, no pending token, no drafts). */
 int pass_reset(pass_ctx *ctx, int seq);
 

@@ -21,6 +21,7 @@ PASS_DBG_DRAFTS, PASS_DBG_PENDING, PASS_DBG_N_ACCEPTED, PASS_DBG_STATUS, PASS_DB
 PASS_MAX_ROWS = 128
 PASS_HOOK_GEMM_STUCK, PASS_HOOK_ATTN_STALE = 0, 1
 PASS_PROMPT_HI_LO, PASS_PROMPT_BF16 = 0, 1
+PASS_TRAIN_LA, PASS_TRAIN_GRAD = 0, 1
 PASS_MAX_TOP_K = 1024
 
 EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_weights", "pass_prefill",
@@ -28,7 +29,8 @@ EXPORTS = ["pass_kv_bytes", "pass_workspace_bytes", "pass_create", "pass_load_we
            "pass_set_top_k", "pass_step_two_call", "pass_debug_schedule",
            "pass_set_kv", "pass_get_kv", "pass_set_state", "pass_get_debug", "pass_last_step_launches",
            "pass_stream", "pass_destroy", "pass_strerror", "pass_debug_linear",
-           "pass_debug_time_linear", "pass_linear_noalloc", "pass_debug_set", "pass_set_prompt_precision"]
+           "pass_debug_time_linear", "pass_linear_noalloc", "pass_debug_set", "pass_set_prompt_precision",
+           "pass_train_workspace_bytes", "pass_train_init", "pass_train_step", "pass_train_get", "pass_train_export"]
 
 
 class PassError(RuntimeError):
@@ -41,6 +43,11 @@ class _Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
                 ("n_layers", "d_model", "n_heads", "d_head", "d_ffn", "vocab", "k_max", "max_batch",
                  "kv_capacity", "dtype")] + [("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
+
+
+class _TrainConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_float) for n in ("lr", "beta1", "beta2", "eps", "weight_decay")] + \
+               [("warmup_steps", ctypes.c_int), ("total_steps", ctypes.c_int)]
 
 
 class _Weights(ctypes.Structure):
@@ -88,6 +95,12 @@ def load_library(path: str = LIB_PATH):
     lib.pass_linear_noalloc.argtypes = [vp, ci, ci, vp, ci, vp]
     lib.pass_debug_set.argtypes = [vp, ci, ci]
     lib.pass_set_prompt_precision.argtypes = [vp, ci]
+    lib.pass_train_workspace_bytes.restype = ctypes.c_size_t
+    lib.pass_train_workspace_bytes.argtypes = [ctypes.POINTER(_Config), ci, ci]
+    lib.pass_train_init.argtypes = [vp, vp, ctypes.c_size_t, ctypes.POINTER(_TrainConfig), ci, ci]
+    lib.pass_train_step.argtypes = [vp, vp, ci, vp, ci, ci, vp]
+    lib.pass_train_get.argtypes = [vp, ci, vp, ctypes.c_size_t]
+    lib.pass_train_export.argtypes = [vp, vp]
     lib.pass_stream.restype = vp
     lib.pass_stream.argtypes = [vp]
     lib.pass_destroy.restype = None
@@ -270,6 +283,34 @@ class PassContext:
         assert y.is_cuda and y.is_contiguous() and y.dtype == self.torch.float32
         _check(self.lib, self.lib.pass_linear_noalloc(self.h, which, layer, x.data_ptr(), x.shape[0], y.data_ptr()))
         return y
+
+    def train_init(self, L: int, max_seqs: int, lr=0.01, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01,
+                   warmup_steps=2000, total_steps=10000) -> None:
+        """pass_train_init: the training workspace is a torch buffer owned by this object."""
+        need = self.lib.pass_train_workspace_bytes(ctypes.byref(self.cfg), L, max_seqs)
+        if need == 0:
+            raise PassError(-1, "unsupported training configuration")
+        self.train_ws = self.torch.empty(need, dtype=self.torch.uint8, device=self.device)
+        hp = _TrainConfig(lr, beta1, beta2, eps, weight_decay, warmup_steps, total_steps)
+        self.train_L = L
+        _check(self.lib, self.lib.pass_train_init(self.h, self.train_ws.data_ptr(), need, ctypes.byref(hp), L, max_seqs))
+
+    def train_step(self, tokens, positions, apply_update: bool = True) -> float:
+        """tokens: [n_seqs][stride] int32 host array, positions: [n_seqs]; returns the batch loss."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        p = np.ascontiguousarray(positions, dtype=np.int32)
+        loss = ctypes.c_float(0.0)
+        _check(self.lib, self.lib.pass_train_step(self.h, t.ctypes.data, t.shape[1], p.ctypes.data, t.shape[0],
+                                                  1 if apply_update else 0, ctypes.byref(loss)))
+        return float(loss.value)
+
+    def train_get(self, what: int) -> np.ndarray:
+        a = np.empty((self.train_L, self.shape.d_model), dtype=np.float32)
+        _check(self.lib, self.lib.pass_train_get(self.h, what, a.ctypes.data, a.nbytes))
+        return a
+
+    def train_export(self, la_emb) -> None:
+        _check(self.lib, self.lib.pass_train_export(self.h, la_emb.data_ptr()))
 
     def set_prompt_precision(self, mode: int) -> None:
         """pass_set_prompt_precision: PASS_PROMPT_HI_LO (default) or PASS_PROMPT_BF16 for long prompts."""

@@ -12,6 +12,7 @@
 #include "gemm_tc.cuh"
 #include "kernels_simt.cuh"
 #include "kernels_verify.cuh"
+#include "train.cuh"
 
 using namespace pass;
 
@@ -163,6 +164,24 @@ struct pass_ctx {
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
     bool use_tc = false;
     bool prompt_plain_bf16 = false;    // pass_set_prompt_precision: long prompts with plain bf16 activations
+    // training of the look-ahead embeddings (pass_train_*): everything lives in the caller's training workspace
+    struct Train {
+        bool ready = false;
+        pass_train_config hp;
+        int L = 0, max_seqs = 0, step = 0, n_max = 0;
+        char* ws = nullptr;
+        std::vector<CUtensorMap> tm_qkv_t, tm_o_t, tm_gu_t, tm_d_t;     // transposed weights, packed
+        CUtensorMap tm_lm_t;
+        float *master = nullptr, *m = nullptr, *v = nullptr, *grad = nullptr;
+        float *h_in = nullptr, *qkv = nullptr, *attn = nullptr, *h_mid = nullptr, *gu = nullptr;   // saved per layer
+        float *h_last = nullptr, *dh = nullptr, *t0 = nullptr, *t1 = nullptr, *dlogits = nullptr, *loss_row = nullptr, *scratch = nullptr;
+        int* targets = nullptr;
+        __nv_bfloat16* stage = nullptr;                                 // hi | lo rows of a GEMM's input, any K
+        std::map<std::pair<int, int>, CUtensorMap> stage_maps;          // by (K, npad)
+        int ng = 0;                                                     // columns of the interleaved gate|up output
+        int* pin_targets = nullptr;
+        float* pin_loss = nullptr;
+    } tr;
     bool packed = false;               // the GEMMs stream the packed copy of the weights (PASS_NO_PACK: the caller's matrices)
     char* d_packed = nullptr;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
@@ -1516,6 +1535,8 @@ void pass_destroy(pass_ctx* c) {
     if (c->pin_states) cudaFreeHost(c->pin_states);
     if (c->pin_status) cudaFreeHost(c->pin_status);
     if (c->pin_tok) cudaFreeHost(c->pin_tok);
+    if (c->tr.pin_targets) cudaFreeHost(c->tr.pin_targets);
+    if (c->tr.pin_loss) cudaFreeHost(c->tr.pin_loss);
     delete c;
 }
 
@@ -1533,3 +1554,261 @@ const char* pass_strerror(int code) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------- look-ahead embedding training
+namespace {
+
+struct TrainLayout {
+    size_t qkv_t, o_t, gu_t, d_t, lm_t;          // per-layer strides are the matrix sizes
+    size_t master, m, v, grad, h_in, qkv, attn, h_mid, gu, h_last, dh, t0, t1, dlogits, loss_row, scratch, targets, stage;
+    size_t total;
+};
+
+TrainLayout make_train_layout(const pass_config& c, int L, int max_seqs) {
+    TrainLayout T;
+    Carve cv;
+    const size_t d = c.d_model, f = c.d_ffn, V = c.vocab, nl = c.n_layers, R = (size_t)L * max_seqs;
+    const size_t ng = ((f + 63) / 64) * 128, wide = std::max(std::max(3 * d, 2 * f), ng);
+    T.qkv_t = cv.take(nl * packed_matrix_bytes(d, 3 * d, 128));
+    T.o_t = cv.take(nl * packed_matrix_bytes(d, d, 128));
+    T.gu_t = cv.take(nl * packed_matrix_bytes(d, 2 * f, 128));
+    T.d_t = cv.take(nl * packed_matrix_bytes(f, d, 128));
+    T.lm_t = cv.take(packed_matrix_bytes(d, V, 128));
+    T.master = cv.take(kMaxLA * d * 4); T.m = cv.take(kMaxLA * d * 4); T.v = cv.take(kMaxLA * d * 4); T.grad = cv.take(kMaxLA * d * 4);
+    T.h_in = cv.take(nl * R * d * 4); T.qkv = cv.take(nl * R * 3 * d * 4); T.attn = cv.take(nl * R * d * 4);
+    T.h_mid = cv.take(nl * R * d * 4); T.gu = cv.take(nl * R * ng * 4);
+    T.h_last = cv.take(R * d * 4); T.dh = cv.take(R * d * 4); T.t0 = cv.take(R * wide * 4); T.t1 = cv.take(R * wide * 4);
+    T.dlogits = cv.take(R * V * 4); T.loss_row = cv.take(R * 4);
+    T.scratch = cv.take((size_t)max_seqs * c.n_heads * 2 * L * (size_t)(c.kv_capacity) * 4);
+    T.targets = cv.take(R * 4);
+    T.stage = cv.take((size_t)2 * kMaxRows * std::max(wide, V) * 2);
+    T.total = cv.off;
+    return T;
+}
+
+// One weight-streaming GEMM of the training passes: y [R][N] = x [R][K] (float32) times the matrix behind the
+// maps, through the hi | lo staging rows.  n_maps = 3: three matrices of seg rows each one after the other (Q, K, V);
+// interleave: gate | up in blocks of 64.
+int train_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2, int seg_tiles,
+               bool interleave, int N, int n_tiles, int K, const float* x, int R, float* y) {
+    const int npad = npad_for(R);
+    auto key = std::make_pair(K, npad);
+    auto it = c->tr.stage_maps.find(key);
+    if (it == c->tr.stage_maps.end()) {
+        CUtensorMap m;
+        if (!make_map(&m, c->tr.stage, 2 * kMaxRows, K, npad)) return PASS_ERR_CUDA;
+        it = c->tr.stage_maps.emplace(key, m).first;
+    }
+    LAUNCH(c, k_split_rows, dim3((K + 255) / 256, R), 256, x, K, c->tr.stage, npad / 2);
+    GemmParams p = gemm_base(c, R, npad, K, n_tiles, N, kEpiLogits);
+    p.packed = 1;
+    p.interleave = interleave ? 1 : 0;
+    if (seg_tiles > 0) p.seg_tiles0 = p.seg_tiles1 = seg_tiles;
+    p.logits = y;
+    launch_gemm(c, a0, a1, a2, it->second, p);
+    return PASS_OK;
+}
+int train_gemm1(pass_ctx* c, const CUtensorMap& a, int N, int K, const float* x, int R, float* y) {
+    return train_gemm(c, a, a, a, 0, false, N, (N + kTileN - 1) / kTileN, K, x, R, y);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pass_train_workspace_bytes(const pass_config* cfg, int L, int max_seqs) {
+    if (!config_ok(cfg) || cfg->dtype != PASS_DTYPE_BF16 || L < 1 || L > cfg->k_max || max_seqs < 1 ||
+        max_seqs > cfg->max_batch || L * max_seqs > kMaxRows)
+        return 0;
+    return make_train_layout(*cfg, L, max_seqs).total;
+}
+
+int pass_train_init(pass_ctx* c, void* train_ws_device, size_t bytes, const pass_train_config* hp, int L, int max_seqs) {
+    if (!c || !train_ws_device || !hp || ((uintptr_t)train_ws_device & 255)) return PASS_ERR_INVALID_ARG;
+    if (!c->weights_loaded || !c->use_tc || !c->packed) return PASS_ERR_STATE;
+    const size_t need = pass_train_workspace_bytes(&c->cfg, L, max_seqs);
+    if (need == 0) return PASS_ERR_INVALID_ARG;
+    if (bytes < need) return PASS_ERR_CAPACITY;
+    if (!(hp->lr > 0.f) || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f) ||
+        !(hp->eps > 0.f) || hp->weight_decay < 0.f || hp->warmup_steps < 0 || hp->total_steps < 1)
+        return PASS_ERR_INVALID_ARG;
+    if (c->pending_collect) {
+        const int rc = pass_step_collect(c, nullptr, nullptr);
+        if (rc != PASS_OK) return rc;
+    }
+    typedef __nv_bfloat16 bf;
+    pass_ctx::Train& t = c->tr;
+    const TrainLayout T = make_train_layout(c->cfg, L, max_seqs);
+    const int d = c->md.d, f = c->md.f, V = c->md.V, nl = c->md.n_layers;
+    char* w = (char*)train_ws_device;
+    t.ws = w; t.hp = *hp; t.L = L; t.max_seqs = max_seqs; t.step = 0; t.n_max = c->md.cap;
+    t.ng = ((f + 63) / 64) * 128;
+    t.master = (float*)(w + T.master); t.m = (float*)(w + T.m); t.v = (float*)(w + T.v); t.grad = (float*)(w + T.grad);
+    t.h_in = (float*)(w + T.h_in); t.qkv = (float*)(w + T.qkv); t.attn = (float*)(w + T.attn); t.h_mid = (float*)(w + T.h_mid);
+    t.gu = (float*)(w + T.gu); t.h_last = (float*)(w + T.h_last); t.dh = (float*)(w + T.dh); t.t0 = (float*)(w + T.t0);
+    t.t1 = (float*)(w + T.t1); t.dlogits = (float*)(w + T.dlogits); t.loss_row = (float*)(w + T.loss_row);
+    t.scratch = (float*)(w + T.scratch); t.targets = (int*)(w + T.targets); t.stage = (bf*)(w + T.stage);
+    t.stage_maps.clear();
+    if (!t.pin_targets && cudaMallocHost((void**)&t.pin_targets, sizeof(int) * kMaxRows) != cudaSuccess) return PASS_ERR_CUDA;
+    if (!t.pin_loss && cudaMallocHost((void**)&t.pin_loss, sizeof(float) * kMaxRows) != cudaSuccess) return PASS_ERR_CUDA;
+    // transposed copies of the weights in streaming order (the backward GEMMs multiply by W, not by its transpose)
+    auto pack_t = [&](CUtensorMap* m, char* dst, const void* s0, const void* s1, const void* s2, int n_src, int rows_src, int N) -> bool {
+        const int K = n_src * rows_src, n_tiles = (N + 127) / 128, kbpt = (K + kBlockK - 1) / kBlockK;
+        PackTSources ps;
+        ps.src[0] = (const bf*)s0; ps.src[1] = (const bf*)s1; ps.src[2] = (const bf*)s2;
+        LAUNCH(c, k_pack_weight_t, n_tiles * kbpt, 128, ps, n_src, rows_src, N, kbpt, (bf*)dst);
+        return make_map_packed(m, dst, (uint64_t)n_tiles * kbpt, 128);
+    };
+    t.tm_qkv_t.resize(nl); t.tm_o_t.resize(nl); t.tm_gu_t.resize(nl); t.tm_d_t.resize(nl);
+    for (int l = 0; l < nl; l++) {
+        if (!pack_t(&t.tm_qkv_t[l], w + T.qkv_t + l * packed_matrix_bytes(d, 3 * d, 128), c->wq[l], c->wk[l], c->wv[l], 3, d, d)) return PASS_ERR_CUDA;
+        if (!pack_t(&t.tm_o_t[l], w + T.o_t + l * packed_matrix_bytes(d, d, 128), c->wo[l], c->wo[l], c->wo[l], 1, d, d)) return PASS_ERR_CUDA;
+        if (!pack_t(&t.tm_gu_t[l], w + T.gu_t + l * packed_matrix_bytes(d, 2 * f, 128), c->wg[l], c->wu[l], c->wu[l], 2, f, d)) return PASS_ERR_CUDA;
+        if (!pack_t(&t.tm_d_t[l], w + T.d_t + l * packed_matrix_bytes(f, d, 128), c->wd[l], c->wd[l], c->wd[l], 1, d, f)) return PASS_ERR_CUDA;
+    }
+    if (!pack_t(&t.tm_lm_t, w + T.lm_t, c->lm_head, c->lm_head, c->lm_head, 1, V, d)) return PASS_ERR_CUDA;
+    // float32 master rows from the context's look-ahead table, moments at zero
+    LAUNCH(c, (k_rows_convert<bf>), (kMaxLA * d + 255) / 256, 256, (const bf*)c->la_emb, t.master, (size_t)c->md.k_max * d, 1);
+    CUDA_TRY(cudaMemsetAsync(t.m, 0, sizeof(float) * kMaxLA * d, c->stream));
+    CUDA_TRY(cudaMemsetAsync(t.v, 0, sizeof(float) * kMaxLA * d, c->stream));
+    CUDA_TRY(cudaMemsetAsync(t.grad, 0, sizeof(float) * kMaxLA * d, c->stream));
+    CHECK_LAUNCHES(c);
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    t.ready = true;
+    return PASS_OK;
+}
+
+static float train_lr(const pass_train_config& hp, int step) {
+    if (hp.warmup_steps > 0 && step < hp.warmup_steps) return hp.lr * (float)(step + 1) / (float)hp.warmup_steps;
+    if (step >= hp.total_steps) return 0.f;
+    const double prog = (double)(step - hp.warmup_steps) / (double)std::max(1, hp.total_steps - hp.warmup_steps);
+    return (float)(0.5 * hp.lr * (1.0 + std::cos(3.14159265358979323846 * prog)));
+}
+
+int pass_train_step(pass_ctx* c, const int32_t* tokens, int stride, const int32_t* positions, int n_seqs, int apply_update,
+                    float* loss_out) {
+    if (!c || !tokens || !positions || !loss_out || n_seqs < 1 || stride < 1) return PASS_ERR_INVALID_ARG;
+    pass_ctx::Train& t = c->tr;
+    if (!t.ready) return PASS_ERR_STATE;
+    if (n_seqs > t.max_seqs) return PASS_ERR_CAPACITY;
+    typedef __nv_bfloat16 bf;
+    const ModelDims& md = c->md;
+    const int L = t.L, R = n_seqs * L, d = md.d, f = md.f, V = md.V, nl = md.n_layers, dt = d / kTileN;
+    for (int b = 0; b < n_seqs; b++) {
+        const int n = positions[b];
+        if (n < 0 || n + 1 + L >= stride) return PASS_ERR_INVALID_ARG;        // the targets w_{n+2} .. w_{n+1+L} must exist
+        if (n + 1 + L > md.cap) return PASS_ERR_CAPACITY;
+        for (int i = 0; i <= n + 1 + L; i++)
+            if (tokens[(size_t)b * stride + i] < 0 || tokens[(size_t)b * stride + i] >= V) return PASS_ERR_INVALID_ARG;
+    }
+    // the prompt part w_0 .. w_n of every sequence: keys and values into the cache, through the prompt pass
+    for (int b = 0; b < n_seqs; b++) {
+        const int rc = pass_prefill(c, b, tokens + (size_t)b * stride, positions[b] + 2);
+        if (rc != PASS_OK) return rc;
+        for (int t_ = 0; t_ < L; t_++) t.pin_targets[b * L + t_] = tokens[(size_t)b * stride + positions[b] + 2 + t_];
+    }
+    CUDA_TRY(cudaMemcpyAsync(t.targets, t.pin_targets, sizeof(int) * R, cudaMemcpyHostToDevice, c->stream));
+    // ---- forward over the look-ahead rows, keeping what the backward pass needs
+    LAUNCH(c, k_train_rows, R, 256, c->d_states, t.master, L, d, c->d_h, c->d_row_seq, c->d_row_pos);
+    LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
+    float* h = c->d_h;
+    int rc = PASS_OK;
+    for (int l = 0; l < nl && rc == PASS_OK; l++) {
+        float* h_in = t.h_in + (size_t)l * R * d; float* qkv = t.qkv + (size_t)l * R * 3 * d;
+        float* attn = t.attn + (size_t)l * R * d; float* h_mid = t.h_mid + (size_t)l * R * d; float* gu = t.gu + (size_t)l * R * t.ng;
+        CUDA_TRY(cudaMemcpyAsync(h_in, h, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, c->stream));
+        LAUNCH(c, (k_rmsnorm<bf>), R, 256, h, (const bf*)c->norm_attn[l], d, md.eps, t.t0);
+        rc = train_gemm(c, c->tm_wq[l], c->tm_wk[l], c->tm_wv[l], dt, false, 3 * d, 3 * dt, d, t.t0, R, qkv);
+        if (rc != PASS_OK) break;
+        LAUNCH(c, (k_rope_kv<bf>), R, 256, qkv, c->d_cs, c->d_row_seq, c->d_row_pos, md, l, (bf*)c->kv_k, (bf*)c->kv_v);
+        if (md.dh == 128)
+            LAUNCH(c, (k_attn_simple<bf, 128, false>), dim3(md.H, R), 128, qkv, 3 * d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)attn, 0);
+        else
+            LAUNCH(c, (k_attn_simple<bf, 64, false>), dim3(md.H, R), 128, qkv, 3 * d, c->d_row_seq, c->d_row_pos, md, l, (const bf*)c->kv_k, (const bf*)c->kv_v, (void*)attn, 0);
+        rc = train_gemm1(c, c->tm_wo[l], d, d, attn, R, t.t0);
+        if (rc != PASS_OK) break;
+        LAUNCH(c, k_add_rows, (R * d + 255) / 256, 256, h, t.t0, (size_t)R * d);
+        CUDA_TRY(cudaMemcpyAsync(h_mid, h, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, c->stream));
+        LAUNCH(c, (k_rmsnorm<bf>), R, 256, h, (const bf*)c->norm_ffn[l], d, md.eps, t.t0);
+        rc = train_gemm(c, c->tm_wg[l], c->tm_wu[l], c->tm_wu[l], 0, true, t.ng, (f + 63) / 64, d, t.t0, R, gu);
+        if (rc != PASS_OK) break;
+        LAUNCH(c, k_swiglu_il, dim3((f + 255) / 256, R), 256, gu, t.ng, f, t.t0);
+        rc = train_gemm1(c, c->tm_wd[l], d, f, t.t0, R, t.t1);
+        if (rc != PASS_OK) break;
+        LAUNCH(c, k_add_rows, (R * d + 255) / 256, 256, h, t.t1, (size_t)R * d);
+    }
+    if (rc != PASS_OK) return rc;
+    CUDA_TRY(cudaMemcpyAsync(t.h_last, h, sizeof(float) * R * d, cudaMemcpyDeviceToDevice, c->stream));
+    LAUNCH(c, (k_rmsnorm<bf>), R, 256, h, (const bf*)c->final_norm, d, md.eps, t.t0);
+    rc = train_gemm1(c, c->tm_lm, V, d, t.t0, R, c->d_logits);
+    if (rc != PASS_OK) return rc;
+    // ---- loss on the look-ahead outputs, gradient with respect to the logits (mean over rows)
+    LAUNCH(c, k_ce_grad, R, 256, c->d_logits, t.targets, V, 1.f / (float)R, t.dlogits, t.loss_row);
+    // ---- backward over the same rows
+    rc = train_gemm1(c, t.tm_lm_t, d, V, t.dlogits, R, t.t0);
+    if (rc != PASS_OK) return rc;
+    LAUNCH(c, (k_rmsnorm_bwd<bf>), R, 256, t.t0, t.h_last, (const bf*)c->final_norm, d, md.eps, (const float*)nullptr, t.dh);
+    for (int l = nl - 1; l >= 0 && rc == PASS_OK; l--) {
+        float* h_in = t.h_in + (size_t)l * R * d; float* qkv = t.qkv + (size_t)l * R * 3 * d;
+        float* h_mid = t.h_mid + (size_t)l * R * d; float* gu = t.gu + (size_t)l * R * t.ng;
+        rc = train_gemm1(c, t.tm_d_t[l], f, d, t.dh, R, t.t0);                       // d act
+        if (rc != PASS_OK) break;
+        LAUNCH(c, k_swiglu_il_bwd, dim3((f + 255) / 256, R), 256, gu, t.ng, f, t.t0, t.t1);   // [d gate | d up]
+        rc = train_gemm1(c, t.tm_gu_t[l], d, 2 * f, t.t1, R, t.t0);                  // d (normalised input of the feed-forward)
+        if (rc != PASS_OK) break;
+        LAUNCH(c, (k_rmsnorm_bwd<bf>), R, 256, t.t0, h_mid, (const bf*)c->norm_ffn[l], d, md.eps, (const float*)t.dh, t.dh);
+        rc = train_gemm1(c, t.tm_o_t[l], d, d, t.dh, R, t.t0);                       // d attention output
+        if (rc != PASS_OK) break;
+        if (md.dh == 128)
+            LAUNCH(c, (k_attn_la_bwd<bf, 128>), dim3(md.H, n_seqs), 128, qkv, t.t0, c->d_states, md, l, L, (const bf*)c->kv_k, (const bf*)c->kv_v, t.scratch, t.n_max, t.t1);
+        else
+            LAUNCH(c, (k_attn_la_bwd<bf, 64>), dim3(md.H, n_seqs), 128, qkv, t.t0, c->d_states, md, l, L, (const bf*)c->kv_k, (const bf*)c->kv_v, t.scratch, t.n_max, t.t1);
+        LAUNCH(c, k_rope_bwd, R, 256, t.t1, c->d_cs, d, md.dh);
+        rc = train_gemm1(c, t.tm_qkv_t[l], d, 3 * d, t.t1, R, t.t0);                 // d (normalised input of attention)
+        if (rc != PASS_OK) break;
+        LAUNCH(c, (k_rmsnorm_bwd<bf>), R, 256, t.t0, h_in, (const bf*)c->norm_attn[l], d, md.eps, (const float*)t.dh, t.dh);
+    }
+    if (rc != PASS_OK) return rc;
+    // ---- gradient of the look-ahead rows (sum over sequences; the 1 / rows factor is in the loss) and the update
+    const float lr = train_lr(t.hp, t.step);
+    const float b1 = 1.f - std::pow(t.hp.beta1, (float)(t.step + 1)), b2 = 1.f - std::pow(t.hp.beta2, (float)(t.step + 1));
+    LAUNCH(c, k_la_grad_adamw, (L * d + 255) / 256, 256, t.dh, n_seqs, L, d, t.grad, t.master, t.m, t.v, lr, t.hp.beta1,
+           t.hp.beta2, t.hp.eps, t.hp.weight_decay, b1, b2, apply_update ? 1 : 0);
+    CUDA_TRY(cudaMemcpyAsync(t.pin_loss, t.loss_row, sizeof(float) * R, cudaMemcpyDeviceToHost, c->stream));
+    CHECK_LAUNCHES(c);
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    const int st = debug_status(c);
+    if (st != PASS_OK) return st;
+    double sum = 0.0;
+    for (int r = 0; r < R; r++) sum += t.pin_loss[r];
+    *loss_out = (float)(sum / R);
+    if (apply_update) t.step++;
+    return PASS_OK;
+}
+
+int pass_train_get(pass_ctx* c, int what, float* dst_host, size_t bytes) {
+    if (!c || !dst_host) return PASS_ERR_INVALID_ARG;
+    pass_ctx::Train& t = c->tr;
+    if (!t.ready) return PASS_ERR_STATE;
+    const size_t n = (size_t)t.L * c->md.d * sizeof(float);
+    if (bytes < n) return PASS_ERR_CAPACITY;
+    const float* src = what == PASS_TRAIN_LA ? t.master : what == PASS_TRAIN_GRAD ? t.grad : nullptr;
+    if (!src) return PASS_ERR_INVALID_ARG;
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    CUDA_TRY(cudaMemcpy(dst_host, src, n, cudaMemcpyDeviceToHost));
+    return PASS_OK;
+}
+
+int pass_train_export(pass_ctx* c, void* la_emb_device) {
+    if (!c || !la_emb_device) return PASS_ERR_INVALID_ARG;
+    pass_ctx::Train& t = c->tr;
+    if (!t.ready) return PASS_ERR_STATE;
+    typedef __nv_bfloat16 bf;
+    LAUNCH(c, (k_rows_convert<bf>), (t.L * c->md.d + 255) / 256, 256, (const bf*)la_emb_device, t.master, (size_t)t.L * c->md.d, 0);
+    CHECK_LAUNCHES(c);
+    CUDA_TRY(cudaStreamSynchronize(c->stream));
+    return PASS_OK;
+}
+
+}  // extern "C"
+
