@@ -57,6 +57,8 @@ WORKLOADS = {
     # the prompt pass by itself (what comes before the first step): prompt tokens per second
     "7b-prefill-2048": dict(shape="7b", k=4, prompt=2048, T=0.0, batch=1, prefill=True),
     "7b-prefill-8192": dict(shape="7b", k=4, prompt=8192, T=0.0, batch=1, prefill=True),
+    # one training step of the look-ahead embeddings: 8 sequences, 4 look-ahead rows, prompts of 512 tokens
+    "7b-la-train-b8-L4-ctx512": dict(shape="7b", k=4, prompt=512, T=0.0, batch=8, train=True),
 }
 
 
@@ -350,6 +352,66 @@ def run_prefill_bench(args, wl, shape):
     ctx.close()
 
 
+def run_train_bench(args, wl, shape):
+    """One training step of the look-ahead embeddings (frozen model, batch of sequences, L look-ahead rows): the
+    prompt parts through the prompt pass, then forward and backward over the B * L look-ahead rows, AdamW.
+    The look-ahead part streams the weights twice (packed copy forward, transposed copy backward): HBM-bound."""
+    import paper_2311_13581_b200 as pb
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    P, B, L = wl["prompt"], wl["batch"], wl["k"]
+    w = si.make_weights(shape, seed=0, device=dev)
+    ctx = pb.PassContext(shape, w, B, P + 64, device=dev)
+    ctx.train_init(L, B)
+    stride = P + L + 8
+    toks = np.stack([np.asarray(si.make_prompt(shape, stride, seq=b), dtype=np.int32) for b in range(B)])
+    pos = [P - 1] * B
+    n = max(1, min(args.steps, 20))
+    for _ in range(max(args.warmup, 3)):
+        ctx.train_step(toks, pos)
+    torch.cuda.synchronize()
+    stream = ctx.stream
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    losses = []
+    with torch.cuda.stream(stream):
+        evs[0].record(stream)
+        for i in range(n):
+            losses.append(ctx.train_step(toks, pos))
+            evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+    ms = evs[0].elapsed_time(evs[-1]) / n
+    # the look-ahead rows alone: a step whose prompts are one token long
+    pos1 = [0] * B
+    for _ in range(3):
+        ctx.train_step(toks, pos1, apply_update=False)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            ctx.train_step(toks, pos1, apply_update=False)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    ms_la = e0.elapsed_time(e1) / n
+    pk, pk_kind = peaks()
+    la_bytes = 2 * weight_bytes(shape)
+    line = {"metric": "look-ahead-embedding training step (7B shape, bf16, frozen model)", "value": B / (ms * 1e-3),
+            "unit": "sequences/s", "n_gpus": 1, "steps": n, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype, "data": "synthetic",
+            "config": {"workload": args.workload, "batch": B, "lookahead": L, "prompt_len": P,
+                       "l2": "weights (13.2 GB forward, 13.2 GB backward) exceed L2"},
+            "per_step_ms": percentiles(per), "loss_first_last": [losses[0], losses[-1]],
+            "lookahead_rows_only_ms": ms_la, "gpu_launches": None,
+            "e2e": {"value": B / (ms * 1e-3), "unit": "sequences/s", "h2d_bytes_per_step": int(toks.nbytes) + 4 * B,
+                    "d2h_bytes_per_step": 4 * B * L, "note": "the timed calls take their tokens from host memory and return the loss to it"},
+            "roofline": {"bound": "hbm", "kernel": "forward + backward over the look-ahead rows (k_gemm_tc on packed and transposed weights)",
+                         "achieved": la_bytes / (ms_la * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "peak_kind": pk_kind, "unit": "GB/s",
+                         "frac": la_bytes / (ms_la * 1e-3) / 1e9 / pk["hbm_gbs"], "traffic": None, "algorithmic_bytes": la_bytes}}
+    print(json.dumps(line))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -368,6 +430,9 @@ def main():
         return
     if wl.get("prefill"):
         run_prefill_bench(args, wl, shape)
+        return
+    if wl.get("train"):
+        run_train_bench(args, wl, shape)
         return
 
     import paper_2311_13581_b200 as pb
