@@ -15,12 +15,11 @@
 //     CTA (one CTA per SM), so every SM pulls the same number of weight bytes whatever N is; with at
 //     least as many tiles as CTAs only the n_tiles mod CTAs odd tiles are streamed and the GEMM ends
 //     on whole tiles (see get_piece).  A tile cut across CTAs is summed in k order - deterministic -
-//     by one CTA, which then runs the fused epilogue.  Which CTA, and how it learns that the parts
-//     are there, depends on the row padding: with 16 rows per half (npad = 32, i.e. 9 to 16 token
-//     rows: k = 4..7 look-ahead tokens at batch 1) it is the CTA holding the tile's first k-blocks,
-//     which finds the other parts in EMPTY-or-value words (no counter, see ll_gather); with any other
-//     padding (1 to 8 rows: k = 0..3; 17 rows and more: k = 8, batches, prompt chunks) it is the LAST
-//     CTA to arrive (counter per tile).
+//     by one CTA, which then runs the fused epilogue: the CTA holding the tile's first k-blocks (that
+//     piece is the last of its own range), which finds the other parts in EMPTY-or-value words (no
+//     counter, see ll_gather).  Up to 16 token rows go through that in one or two passes of nine rows;
+//     more rows (k = 8, batches) sixteen at a time.  (The prompt-chunk instantiation computes every unit
+//     whole and shares nothing.)
 //   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 1 TMEM allocation + MMA issue,
 //     warps 2-5 epilogue (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue
 //     of one piece overlaps the main loop of the next.
@@ -65,8 +64,8 @@ struct GemmParams {
     int stages;
     int epi;
     int n_out;                     // output features in total
-    float* partial_ws;             // [gridDim][2][rh][128] fp32: rh != 16 (arrival counter per tile)
-    float* ll_ws;                  // [gridDim][2][16][128] fp32 words, EMPTY between launches: rh == 16 (9..16 rows)
+    float* partial_ws;             // [gridDim][2][rows][128] fp32 + arrival counter per tile: prompt-chunk instantiation only
+    float* ll_ws;                  // [gridDim][2][rh][128] fp32 words, EMPTY between launches: every launch of the step's kernel
     int* tile_counters;            // [n_tiles], zero between launches
     int* status;
     // rstd of the input rows (epilogues that follow an RMSNorm): parts [n_parts_in][kRowsCap]
@@ -430,7 +429,7 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
     }
 }
 
-// With 16 rows per half (9 to 16 token rows) partial sums are handed over without a counter: a slot word is either EMPTY (all
+// Partial sums are handed over without a counter: a slot word is either EMPTY (all
 // bits set - a NaN pattern that fp32 arithmetic never produces, it makes the canonical 0x7fffffff) or a
 // value.  Contributors just store their values; the finisher loads the words it needs and repeats the
 // load until none of them is empty; when it is done with a tile it stores EMPTY back, so every launch
@@ -453,6 +452,7 @@ constexpr int kLLPeers = 5;         // other contributors fetched per trip
 // acc[j] += value of row row0 + j from each of `n_others` contributors (slots `first` + q * stride, k order),
 // for this thread's feature.  Spins (bounded) until no word is EMPTY, then marks the words EMPTY again if
 // `reset`.  Returns false on time-out.
+template <int kLLRows>
 __device__ __forceinline__ bool ll_gather(float* first, size_t stride, int n_others, int row0, int nrows,
                                           float (&acc)[kLLRows], volatile int* s_abort, int* g_status) {
     bool fine = true;
@@ -905,14 +905,70 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                                 cs9[j] = c0 == 0 ? cs_pre[j] : (j < 16 - kLLRows ? cs_pre[kLLRows + j] : make_float2(0.f, 0.f));
                             }
                             if (!whole)
-                                ll_gather(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
+                                ll_gather<kLLRows>(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
                             if (et == 0 && c0 == 0 && !whole) PASS_TRACE(oi, 5);
                             epi_store<kLLRows, BIG>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
                                                p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs9 : nullptr);
                         }
                         if (!whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
                     }
-                } else {
+                } else if (!BIG && has_lo) {
+                    // More than 16 token rows (k = 8, batches): the same counter-free hand-over, sixteen rows at a
+                    // time, each group as two passes of eight rows through the epilogue.
+                    const bool contributor = !whole && pc.index != 0;
+                    float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
+                    const size_t peer_stride = 2 * slot_floats;
+                    const int n = pc.tile * kTileN + ec.lane_in_tile;
+                    if (p.epi == kEpiResid) g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
+                    if (!contributor) tile_done = true;
+#pragma unroll 1
+                    for (int rg = 0; rg < p.rh; rg += 16) {
+                        float av[16];
+#pragma unroll
+                        for (int c0 = 0; c0 < 16; c0 += 8) {
+                            float hi[8], lo[8];
+                            if (rg + c0 < p.rh) {
+                                tmem_ld8(t_addr + rg + c0, hi);
+                                tmem_ld8(t_addr + p.rh + rg + c0, lo);
+                                tmem_ld_wait();
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; j++) av[c0 + j] = rg + c0 < p.rh ? hi[j] + lo[j] : 0.f;
+                        }
+                        if (rg + 16 >= p.rh) {              // the accumulator has been read out: the MMA warp may have it back
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+                        }
+                        if (rg >= p.R) continue;
+                        if (contributor) {
+                            float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
+#pragma unroll
+                            for (int j = 0; j < 16; j++)
+                                if (rg + j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)(rg + j) * kTileN, __float_as_uint(av[j]));
+                            continue;
+                        }
+                        float hv[16];
+#pragma unroll
+                        for (int j = 0; j < 16; j++)
+                            hv[j] = (p.epi == kEpiResid && rg + j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)(rg + j) * p.n_out + n) : 0.f;
+#pragma unroll 1
+                        for (int c0 = 0; c0 < 16; c0 += 8) {
+                            if (rg + c0 >= p.R) break;
+                            float a8[8], h8[8];
+#pragma unroll
+                            for (int j = 0; j < 8; j++) {
+                                a8[j] = c0 == 0 ? av[j] : av[8 + j];
+                                h8[j] = c0 == 0 ? hv[j] : hv[8 + j];
+                            }
+                            if (!whole)
+                                ll_gather<8>(peer, peer_stride, pc.n_pieces - 1, rg + c0, min(p.R - rg - c0, 8), a8, &s_abort, cp.status);
+                            epi_store<8, BIG>(p, ec, pc.tile, rg + c0, a8, p.epi == kEpiResid ? h8 : nullptr,
+                                              p.epi == kEpiResid ? &g_pre : nullptr, nullptr);
+                        }
+                    }
+                    if (!contributor && !whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
+                } else if (BIG) {               // prompt chunks (the step's kernel never gets here: it has hi | lo rows)
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
                 // Whole tiles of many rows (prompt chunks): what the residual epilogue reads is requested one
                 // group of eight rows ahead, so that a group does not begin with a trip to L2.

@@ -19,7 +19,7 @@ using namespace pass;
 namespace {
 
 constexpr int kMaxCtas = 160;      // upper bound of CTAs of one GEMM launch (one per SM)
-constexpr size_t kLLRegionBytes = (size_t)(kMaxCtas + 1) * 2 * 16 * 128 * 4;   // per GEMM of a chain; +1: CTA c reads c+1..
+constexpr size_t kLLRegionBytes = (size_t)(kMaxCtas + 1) * 2 * kMaxRows * 128 * 4;   // per GEMM of a chain (rows per half up to 128); +1: CTA c reads c+1..
 
 struct Carve {
     size_t off = 0;

@@ -141,10 +141,9 @@ def test_changing_k_and_temperature_between_steps(tiny_w):
 
 
 def test_bf16_changing_k_alternates_between_the_two_partial_sum_protocols():
-    """k = 4 (9 rows, padded to 16 per half: partial sums handed over through EMPTY-or-value words) and
-    k = 0, 1, 2 (1, 3, 5 rows) or k = 8 (17 rows), which use arrival counters, in one context, back and
-    forth: each protocol must find its scratch as it left it, and the graphs of the different k must not
-    disturb each other."""
+    """k = 4, 1, 0, 2 (up to 16 rows: one group of the counter-free hand-over) and k = 8 (17 rows: two groups)
+    in one context, back and forth: every launch must find the hand-over words EMPTY as the one before left
+    them, and the graphs of the different k must not disturb each other."""
     from parity_util import lockstep, make_pair
     prompt = si.make_prompt(TINY_BF16, 40)
     ctx, oracles, _ = make_pair(TINY_BF16, 1, 400, [prompt], seed=1)
