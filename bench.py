@@ -57,6 +57,7 @@ WORKLOADS = {
     # the prompt pass by itself (what comes before the first step): prompt tokens per second
     "7b-prefill-2048": dict(shape="7b", k=4, prompt=2048, T=0.0, batch=1, prefill=True),
     "7b-prefill-8192": dict(shape="7b", k=4, prompt=8192, T=0.0, batch=1, prefill=True),
+    "7b-l2-prefill-2048": dict(shape="7b", k=4, prompt=2048, T=0.0, batch=1, prefill=True, n_layers=2),   # small enough for ncu
     # one training step of the look-ahead embeddings: 8 sequences, 4 look-ahead rows, prompts of 512 tokens
     "7b-la-train-b8-L4-ctx512": dict(shape="7b", k=4, prompt=512, T=0.0, batch=8, train=True),
 }
@@ -420,6 +421,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b-k4-ctx512-greedy", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the brief runs of the other 7B configurations")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     shape = si.SHAPES[wl["shape"]]
@@ -548,6 +550,33 @@ def main():
         n_chain = 64
         chain_us = min(ctx.debug_time_linear(9, B * (1 + 2 * k), n_chain) for _ in range(3)) * 1e3 / n_chain
 
+    # ---- the other single-sequence configurations of the same model, briefly (default workload, one GPU only):
+    # the look-ahead sweep at a prompt of 2048 tokens and T = 0.8, and a prompt of 8192 tokens at T = 1.0
+    sweep = None
+    if args.workload == "7b-k4-ctx512-greedy" and world == 1 and not args.no_sweep:
+        ctx.close()
+        ctx = None
+        sweep = []
+        for P2, T2, ks in ((2048, 0.8, (1, 2, 4, 6, 8)), (8192, 1.0, (4,))):
+            c2 = pb.PassContext(shape, w, 1, P2 + 60 * 9 * len(ks) + 64, device=dev)
+            c2.prefill(0, si.make_prompt(shape, P2, seq=7))
+            for k2 in ks:
+                u2 = torch.stack([si.step_uniforms(3, 0, s_, 2 * k2 + 1) for s_ in range(60)]).reshape(60, 1, 2 * k2 + 1).to(dev)
+                for s_ in range(10):
+                    c2.step_enqueue(k2, T2, u2[s_])
+                c2.step_collect()
+                l0 = c2.get_debug(pb.PASS_DBG_KV_LEN).copy()
+                barrier()
+                ms2, _, _, _ = timed_steps(c2, c2.stream, k2, T2, u2, 10, 50, barrier)
+                c2.step_collect()
+                l1 = c2.get_debug(pb.PASS_DBG_KV_LEN).copy()
+                by = weight_bytes(shape) + float(l0.mean() + l1.mean()) / 2 * kv_bytes_per_pos(shape)
+                sweep.append({"k_lookahead": k2, "rows_per_step": 1 + 2 * k2, "prompt_len": P2, "temperature": T2,
+                              "ms_per_step": ms2 / 50, "tokens_per_step": float((l1 - l0).sum()) / 50,
+                              "frac_of_8tbs": by / (ms2 / 50 * 1e-3) / 8e12,
+                              "target_ms_per_step": by / (0.70 * 8e12) * 1e3})
+            c2.close()
+
     ms_total, e2e_ms, tokens, tok_e2e = aggregate_replicas(ms_total, e2e_s * 1e3, tokens, tok_e2e, world, dev)
     if rank != 0:
         return
@@ -580,6 +609,8 @@ def main():
                           "achieved": gbs, "peak": pk["hbm_gbs"], "peak_kind": pk_kind, "unit": "GB/s",
                           "frac": gbs / pk["hbm_gbs"], "algorithmic_bytes": bytes_step},
     }
+    if sweep is not None:
+        line["config_sweep"] = sweep
     if e2e_sampled is not None:
         line["e2e_sampled"] = e2e_sampled
     if k0 is not None:
@@ -600,7 +631,8 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(shape, w, wl, tokens / args.steps)
     print(json.dumps(line))
-    ctx.close()
+    if ctx is not None:
+        ctx.close()
 
 
 def cpu_baseline(shape, w, wl, tokens_per_gpu_step):
