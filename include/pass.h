@@ -291,6 +291,9 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_TRACE         9  /* uint64 [launch][4 GEMMs][CTAs][8]: %globaltimer stamps of the GEMM-chain
                                      launches since the last read, when PASS_TRACE is set in the environment:
                                      activations available, first tile ready, last MMA issued, epilogues done */
+#define PASS_DBG_FOOTPRINT    10  /* int32 [6]: shared memory in bytes of the step's GEMM kernel (static, dynamic at 9..16
+                                     rows) and of its attention kernel (static, dynamic), the SM's total and what the
+                                     system reserves per block: the two kernels are meant to fit on one SM together */
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
 /*

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libpass_b200.so")
 
 PASS_DBG_LOGITS, PASS_DBG_DRAFT_LOGITS, PASS_DBG_KV_LEN, PASS_DBG_N_DRAFT = 0, 1, 2, 3
 PASS_DBG_DRAFTS, PASS_DBG_PENDING, PASS_DBG_N_ACCEPTED, PASS_DBG_STATUS, PASS_DBG_HIDDEN = 4, 5, 6, 7, 8
+PASS_DBG_FOOTPRINT = 10
 PASS_MAX_ROWS = 128
 PASS_HOOK_GEMM_STUCK, PASS_HOOK_ATTN_STALE = 0, 1
 PASS_PROMPT_HI_LO, PASS_PROMPT_BF16 = 0, 1
@@ -260,6 +261,8 @@ class PassContext:
             a = np.empty((B, km), dtype=np.int32)
         elif what == PASS_DBG_STATUS:
             a = np.empty(1, dtype=np.int32)
+        elif what == PASS_DBG_FOOTPRINT:
+            a = np.empty(6, dtype=np.int32)
         else:
             a = np.empty(B, dtype=np.int32)
         _check(self.lib, self.lib.pass_get_debug(self.h, what, a.ctypes.data, a.nbytes))

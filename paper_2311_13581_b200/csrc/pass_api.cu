@@ -1271,6 +1271,27 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         c->trace_launch = 0;
         return PASS_OK;
     }
+    if (what == PASS_DBG_FOOTPRINT) {
+        // shared memory of the step's two big kernels (bf16 models): they are meant to share an SM
+        if (!need(6 * 4)) return PASS_ERR_CAPACITY;
+        if (!c->use_tc) return PASS_ERR_STATE;
+        cudaFuncAttributes ag, aa;
+        CUDA_TRY(cudaFuncGetAttributes(&ag, k_gemm_tc));
+        if (c->md.dh == 128) CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<128, 1, true>));
+        else CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<64, 1, true>));
+        int dev = 0, sm_total = 0, reserved = 0;
+        CUDA_TRY(cudaGetDevice(&dev));
+        CUDA_TRY(cudaDeviceGetAttribute(&sm_total, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
+        CUDA_TRY(cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev));
+        int* o = (int*)dst;
+        o[0] = (int)ag.sharedSizeBytes;
+        o[1] = gemm_stages(32) * (kATileBytes + 32 * 128) + 1024;
+        o[2] = (int)aa.sharedSizeBytes;
+        o[3] = 2 * kAttnStages * kAttnBK * c->md.dh * 2;
+        o[4] = sm_total;
+        o[5] = reserved;
+        return PASS_OK;
+    }
     if (what == PASS_DBG_STATUS) {
         if (!need(4)) return PASS_ERR_CAPACITY;
         CUDA_TRY(cudaMemcpy(dst, c->d_status, 4, cudaMemcpyDeviceToHost));

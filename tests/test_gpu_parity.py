@@ -32,6 +32,18 @@ def test_library_loaded_and_device_is_blackwell():
     assert torch.cuda.get_device_capability(0)[0] == 10
 
 
+def test_gemm_and_attention_ctas_fit_on_one_sm_together():
+    """The attention kernel's CTA and the CTA of the GEMM launch after it are meant to be resident side by
+    side (the GEMM launch streams weights while attention runs: 0.12 ms of a 3.06 ms step at the 7B shape).
+    Their shared memory fills an SM to within a few hundred bytes, so the sum is checked here."""
+    pb = _pb()
+    shape = dataclasses.replace(TINY_BF16, d_head=128, n_heads=2)       # heads of 128, as in the 7B and 13B shapes
+    ctx = pb.PassContext(shape, si.weights_to(si.make_weights(shape, seed=1), "cuda:0"), 1, 64)
+    g_static, g_dyn, a_static, a_dyn, sm_total, reserved = [int(x) for x in ctx.get_debug(pb.PASS_DBG_FOOTPRINT)]
+    assert g_static + g_dyn + reserved + a_static + a_dyn + reserved <= sm_total, (g_static, g_dyn, a_static, a_dyn, sm_total, reserved)
+    ctx.close()
+
+
 # ------------------------------------------------------------------ config 1: tiny fp32
 @pytest.mark.parametrize("T", [0.0, 1.0])
 def test_tiny_fp32_lockstep_k2(tiny_w, T):
