@@ -178,6 +178,7 @@ struct pass_ctx {
         int* targets = nullptr;
         __nv_bfloat16* stage = nullptr;                                 // hi | lo rows of a GEMM's input, any K
         std::map<std::pair<int, int>, CUtensorMap> stage_maps;          // by (K, npad)
+        std::map<int, cudaGraphExec_t> graphs;                          // forward + backward over the look-ahead rows, by batch size
         int ng = 0;                                                     // columns of the interleaved gate|up output
         int* pin_targets = nullptr;
         float* pin_loss = nullptr;
@@ -1551,6 +1552,7 @@ void pass_destroy(pass_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+    for (auto& g : c->tr.graphs) cudaGraphExecDestroy(g.second);
     if (c->pin_params) cudaFreeHost(c->pin_params);
     if (c->pin_unif) cudaFreeHost(c->pin_unif);
     if (c->pin_states) cudaFreeHost(c->pin_states);
@@ -1670,6 +1672,8 @@ int pass_train_init(pass_ctx* c, void* train_ws_device, size_t bytes, const pass
     t.t1 = (float*)(w + T.t1); t.dlogits = (float*)(w + T.dlogits); t.loss_row = (float*)(w + T.loss_row);
     t.scratch = (float*)(w + T.scratch); t.targets = (int*)(w + T.targets); t.stage = (bf*)(w + T.stage);
     t.stage_maps.clear();
+    for (auto& g : t.graphs) cudaGraphExecDestroy(g.second);
+    t.graphs.clear();
     if (!t.pin_targets && cudaMallocHost((void**)&t.pin_targets, sizeof(int) * kMaxRows) != cudaSuccess) return PASS_ERR_CUDA;
     if (!t.pin_loss && cudaMallocHost((void**)&t.pin_loss, sizeof(float) * kMaxRows) != cudaSuccess) return PASS_ERR_CUDA;
     // transposed copies of the weights in streaming order (the backward GEMMs multiply by W, not by its transpose)
@@ -1699,36 +1703,13 @@ int pass_train_init(pass_ctx* c, void* train_ws_device, size_t bytes, const pass
     return PASS_OK;
 }
 
-static float train_lr(const pass_train_config& hp, int step) {
-    if (hp.warmup_steps > 0 && step < hp.warmup_steps) return hp.lr * (float)(step + 1) / (float)hp.warmup_steps;
-    if (step >= hp.total_steps) return 0.f;
-    const double prog = (double)(step - hp.warmup_steps) / (double)std::max(1, hp.total_steps - hp.warmup_steps);
-    return (float)(0.5 * hp.lr * (1.0 + std::cos(3.14159265358979323846 * prog)));
-}
-
-int pass_train_step(pass_ctx* c, const int32_t* tokens, int stride, const int32_t* positions, int n_seqs, int apply_update,
-                    float* loss_out) {
-    if (!c || !tokens || !positions || !loss_out || n_seqs < 1 || stride < 1) return PASS_ERR_INVALID_ARG;
-    pass_ctx::Train& t = c->tr;
-    if (!t.ready) return PASS_ERR_STATE;
-    if (n_seqs > t.max_seqs) return PASS_ERR_CAPACITY;
+// Forward and backward over the look-ahead rows of n_seqs sequences (everything between the prompt passes and
+// the update): enqueued on the context's stream, directly or into a graph capture.
+static int train_enqueue_rows(pass_ctx* c, int n_seqs) {
     typedef __nv_bfloat16 bf;
+    pass_ctx::Train& t = c->tr;
     const ModelDims& md = c->md;
     const int L = t.L, R = n_seqs * L, d = md.d, f = md.f, V = md.V, nl = md.n_layers, dt = d / kTileN;
-    for (int b = 0; b < n_seqs; b++) {
-        const int n = positions[b];
-        if (n < 0 || n + 1 + L >= stride) return PASS_ERR_INVALID_ARG;        // the targets w_{n+2} .. w_{n+1+L} must exist
-        if (n + 1 + L > md.cap) return PASS_ERR_CAPACITY;
-        for (int i = 0; i <= n + 1 + L; i++)
-            if (tokens[(size_t)b * stride + i] < 0 || tokens[(size_t)b * stride + i] >= V) return PASS_ERR_INVALID_ARG;
-    }
-    // the prompt part w_0 .. w_n of every sequence: keys and values into the cache, through the prompt pass
-    for (int b = 0; b < n_seqs; b++) {
-        const int rc = pass_prefill(c, b, tokens + (size_t)b * stride, positions[b] + 2);
-        if (rc != PASS_OK) return rc;
-        for (int t_ = 0; t_ < L; t_++) t.pin_targets[b * L + t_] = tokens[(size_t)b * stride + positions[b] + 2 + t_];
-    }
-    CUDA_TRY(cudaMemcpyAsync(t.targets, t.pin_targets, sizeof(int) * R, cudaMemcpyHostToDevice, c->stream));
     // ---- forward over the look-ahead rows, keeping what the backward pass needs
     LAUNCH(c, k_train_rows, R, 256, c->d_states, t.master, L, d, c->d_h, c->d_row_seq, c->d_row_pos);
     LAUNCH(c, k_rope_table, R, 64, c->d_row_pos, c->d_invfreq, md.dh / 2, c->d_cs);
@@ -1790,6 +1771,63 @@ int pass_train_step(pass_ctx* c, const int32_t* tokens, int stride, const int32_
         LAUNCH(c, (k_rmsnorm_bwd<bf>), R, 256, t.t0, h_in, (const bf*)c->norm_attn[l], d, md.eps, (const float*)t.dh, t.dh);
     }
     if (rc != PASS_OK) return rc;
+    return PASS_OK;
+}
+
+static float train_lr(const pass_train_config& hp, int step) {
+    if (hp.warmup_steps > 0 && step < hp.warmup_steps) return hp.lr * (float)(step + 1) / (float)hp.warmup_steps;
+    if (step >= hp.total_steps) return 0.f;
+    const double prog = (double)(step - hp.warmup_steps) / (double)std::max(1, hp.total_steps - hp.warmup_steps);
+    return (float)(0.5 * hp.lr * (1.0 + std::cos(3.14159265358979323846 * prog)));
+}
+
+int pass_train_step(pass_ctx* c, const int32_t* tokens, int stride, const int32_t* positions, int n_seqs, int apply_update,
+                    float* loss_out) {
+    if (!c || !tokens || !positions || !loss_out || n_seqs < 1 || stride < 1) return PASS_ERR_INVALID_ARG;
+    pass_ctx::Train& t = c->tr;
+    if (!t.ready) return PASS_ERR_STATE;
+    if (n_seqs > t.max_seqs) return PASS_ERR_CAPACITY;
+    typedef __nv_bfloat16 bf;
+    const ModelDims& md = c->md;
+    const int L = t.L, R = n_seqs * L, d = md.d, f = md.f, V = md.V, nl = md.n_layers, dt = d / kTileN;
+    for (int b = 0; b < n_seqs; b++) {
+        const int n = positions[b];
+        if (n < 0 || n + 1 + L >= stride) return PASS_ERR_INVALID_ARG;        // the targets w_{n+2} .. w_{n+1+L} must exist
+        if (n + 1 + L > md.cap) return PASS_ERR_CAPACITY;
+        for (int i = 0; i <= n + 1 + L; i++)
+            if (tokens[(size_t)b * stride + i] < 0 || tokens[(size_t)b * stride + i] >= V) return PASS_ERR_INVALID_ARG;
+    }
+    // the prompt part w_0 .. w_n of every sequence: keys and values into the cache, through the prompt pass
+    for (int b = 0; b < n_seqs; b++) {
+        const int rc = pass_prefill(c, b, tokens + (size_t)b * stride, positions[b] + 2);
+        if (rc != PASS_OK) return rc;
+        for (int t_ = 0; t_ < L; t_++) t.pin_targets[b * L + t_] = tokens[(size_t)b * stride + positions[b] + 2 + t_];
+    }
+    CUDA_TRY(cudaMemcpyAsync(t.targets, t.pin_targets, sizeof(int) * R, cudaMemcpyHostToDevice, c->stream));
+    // ---- forward and backward over the look-ahead rows: one CUDA graph per batch size
+    int rc = PASS_OK;
+    if (c->use_graph) {
+        auto it = t.graphs.find(n_seqs);
+        if (it == t.graphs.end()) {
+            cudaGraph_t g = nullptr;
+            CUDA_TRY(cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+            rc = train_enqueue_rows(c, n_seqs);
+            const cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+            if (rc != PASS_OK || e != cudaSuccess || !g || launch_failed(c)) {
+                if (g) cudaGraphDestroy(g);
+                return rc != PASS_OK ? rc : PASS_ERR_CUDA;
+            }
+            cudaGraphExec_t ge = nullptr;
+            const cudaError_t e2 = cudaGraphInstantiate(&ge, g, 0);
+            cudaGraphDestroy(g);
+            if (e2 != cudaSuccess) return PASS_ERR_CUDA;
+            it = t.graphs.emplace(n_seqs, ge).first;
+        }
+        CUDA_TRY(cudaGraphLaunch(it->second, c->stream));
+    } else {
+        rc = train_enqueue_rows(c, n_seqs);
+        if (rc != PASS_OK) return rc;
+    }
     // ---- gradient of the look-ahead rows (sum over sequences; the 1 / rows factor is in the loss) and the update
     const float lr = train_lr(t.hp, t.step);
     const float b1 = 1.f - std::pow(t.hp.beta1, (float)(t.step + 1)), b2 = 1.f - std::pow(t.hp.beta2, (float)(t.step + 1));
