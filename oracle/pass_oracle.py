@@ -8,8 +8,8 @@ What it holds, each part written from the paper in float64:
 
 * ``TransformerBackend``  - the decoder forward (C, ``pass_oracle.c``) behind a
   tiny "rows in, logits out" interface with a KV cache that can be truncated
-  ("We use the KV cache and update it after every model call according to the
-  number of drafted tokens and the number of accepted tokens", Baselines).
+  (section "Baselines": after each model call the cache is cut back to what the
+  accepted tokens need).
 * ``softmax_T``, ``invcdf``, ``verify`` - the speculative-sampling rule of
   Algorithm 1 / Algorithm 2: accept draft t when r < min(1, target/draft), else
   sample from the positive part of (target - draft) and stop; if every draft is
