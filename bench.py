@@ -42,6 +42,7 @@ WORKLOADS = {
     "tiny-k2-ctx32": dict(shape="tiny", k=2, prompt=32, T=1.0, batch=1),
     # depth-reduced 7B (same layer shape, 4 layers): small enough for multi-pass ncu captures
     "7b-l4-k4-ctx512-greedy": dict(shape="7b", k=4, prompt=512, T=0.0, batch=1, n_layers=4),
+    "7b-l4-k4-ctx8192-T1.0": dict(shape="7b", k=4, prompt=8192, T=1.0, batch=1, n_layers=4),     # long cache, small enough for ncu
     "7b-k0-ctx512-greedy": dict(shape="7b", k=0, prompt=512, T=0.0, batch=1),
     # the sampler of the paper's experiments: top-k 10, temperature 0.8
     "7b-k4-ctx512-T0.8-top10": dict(shape="7b", k=4, prompt=512, T=0.8, batch=1, top_k=10),

@@ -38,6 +38,7 @@ struct AttnParams {
     int debug_stale;               // test hook: the early part pretends the tables said len - debug_stale
     int out_tile_rows;             // > 0: output rows are laid out in token tiles of this many rows, hi rows of a tile
                                    // followed by its lo rows (the layout the next GEMM of a prompt chunk reads)
+    int* status;                   // kStatusTimeout is raised here (k_attn_tc, the only attention kernel that waits)
     int rows_per_block;            // 0: blockIdx.y = sequence, M rows each (a decode step).  > 0: ONE sequence of M rows
                                    // (a prompt chunk), blockIdx.y = block of rows_per_block rows - causal flash attention
 };
@@ -68,16 +69,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // Merge of the slices of one (sequence, head) by the CTA that delivered last.  NS = most slices this
-// instance handles, EB = output elements per thread and batch.  The first batch of partial outputs and
+// instance handles, EB = output elements per thread and batch, NT = threads of the CTA.  The first batch of partial outputs and
 // the (max, sum) pairs are requested together, before anything waits: for the usual case (up to 4 slices,
 // up to 12 rows of 128) the whole merge is one trip to L2.
-template <int DH, int NS, int EB>
+template <int DH, int NS, int EB, int NT = 128>
 __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int row0, int head, float* sm_f) {
     const int tid = threadIdx.x, M = p.M;
     auto load_batch = [&](int base, float (&vals)[EB][NS]) {
 #pragma unroll
         for (int e = 0; e < EB; e++) {
-            const int idx = min(base + e * 128 + tid, M * DH - 1);
+            const int idx = min(base + e * NT + tid, M * DH - 1);
             const int i = idx / DH, dcol = idx % DH;
 #pragma unroll
             for (int sidx = 0; sidx < NS; sidx++)
@@ -86,7 +87,7 @@ __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int r
     };
     float vals[EB][NS];
     load_batch(0, vals);
-    for (int i = tid; i < M; i += 128) {
+    for (int i = tid; i < M; i += NT) {
         float2 ml[NS];
 #pragma unroll
         for (int sidx = 0; sidx < NS; sidx++)
@@ -107,11 +108,11 @@ __device__ __forceinline__ void attn_merge(const AttnParams& p, size_t hb, int r
             if (sidx < p.n_split) sm_f[sidx * 32 + i] = f[sidx] * inv;
     }
     __syncthreads();
-    for (int base = 0; base < M * DH; base += 128 * EB) {
+    for (int base = 0; base < M * DH; base += NT * EB) {
         if (base > 0) load_batch(base, vals);
 #pragma unroll
         for (int e = 0; e < EB; e++) {
-            const int idx = base + e * 128 + tid;
+            const int idx = base + e * NT + tid;
             if (idx < M * DH) {
                 const int i = idx / DH, dcol = idx % DH;
                 float v = 0.f;

@@ -10,6 +10,7 @@
 
 #include "attn_fd.cuh"
 #include "gemm_tc.cuh"
+#include "attn_tc.cuh"
 #include "kernels_simt.cuh"
 #include "kernels_verify.cuh"
 #include "train.cuh"
@@ -153,6 +154,9 @@ struct pass_ctx {
     bool use_pdl = true;
     bool attn_long = false;       // this step's contexts are long: twice as many attention slices (see step_launch)
     int attn_long_from = 3072;    // PASS_ATTN_LONG_FROM: cached positions from which a step counts as long
+    bool attn_tc = true;          // PASS_ATTN_NO_TC: long contexts keep the mma.sync kernel (k_attn_tc otherwise, d_head 128, <= 16 rows)
+    bool attn_tc_ready = false, attn_tc_smem_set = false;
+    AttnTcMaps attn_tc_maps;      // the key and the value cache as matrices of 128 columns
     bool attn_cluster = true;     // PASS_ATTN_NO_CLUSTER: merge attention slices through global memory
     int attn_debug_stale = 0;     // pass_debug_set(PASS_HOOK_ATTN_STALE, n): attention's early part works from a cache length n short
     int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
@@ -506,6 +510,27 @@ static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     c->launches++;
 }
 
+// Long caches, d_head 128, at most 16 rows per sequence: scores on tcgen05 (attn_tc.cuh), one CTA per SM.
+static void launch_attn_tc(pass_ctx* c, const AttnParams& ap, int n_seq) {
+    if (!c->attn_tc_smem_set) {
+        note_err(c, cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem), "k_attn_tc shared memory size");
+        c->attn_tc_smem_set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->md.H, n_seq, ap.n_split);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = c->use_pdl ? 1 : 0;
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_tc, c->attn_tc_maps, ap), "k_attn_tc launch");
+    c->launches++;
+}
+
 // Can the slices of every (sequence, head) run as one cluster each, all at the same time?  Asked once per
 // context, kernel instance, slice count and batch; if not (or with more than 8 slices) the merge goes through
 // global memory.
@@ -670,13 +695,18 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
         const bool plain = big && c->prompt_plain_bf16;
         ap.out = c->d_attn_bf; ap.lo_row0 = plain ? -1 : rh; ap.debug_stale = c->attn_debug_stale;
         ap.rows_per_block = 0;
+        ap.status = c->d_status;
         ap.out_tile_rows = big && !plain ? rh : 0;
-        if (M <= 32) {
+        if (M <= 16 && md.dh == kTcDH && c->attn_long && c->attn_tc && c->attn_tc_ready) {
+            ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
+            launch_attn_tc(c, ap, n_seq);
+        } else if (M <= 32) {
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             // Long contexts: the key loop (tensor-core work of 4 warps) outweighs everything that one CTA per
             // SM buys at short contexts, so the slices are doubled - two CTAs per SM, 8 warps on the keys.
             if (c->attn_long && ap.n_split * 2 <= 8) ap.n_split *= 2;
+            if (const char* e = getenv("PASS_ATTN_SPLIT")) ap.n_split = std::max(1, std::min(std::min(kAttnMaxSplit, 2 * kMaxCtas / (md.H * n_seq)), atoi(e)));
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
             else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
         } else {
@@ -860,6 +890,12 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
         c->use_tc = getenv("PASS_FORCE_SIMT") == nullptr;
         c->use_pdl = getenv("PASS_NO_PDL") == nullptr;
         c->attn_cluster = getenv("PASS_ATTN_NO_CLUSTER") == nullptr;
+        c->attn_tc = getenv("PASS_ATTN_NO_TC") == nullptr;
+        if (c->md.dh == kTcDH) {
+            const uint64_t cache_rows = (uint64_t)c->md.n_layers * c->md.B * c->md.H * c->md.cap;
+            c->attn_tc_ready = cache_rows < (1ull << 31) && make_map(&c->attn_tc_maps.k, kv_k, cache_rows, kTcDH, kTcBK) &&
+                               make_map(&c->attn_tc_maps.v, kv_v, cache_rows, kTcDH, kTcBK);
+        }
         if (const char* e = getenv("PASS_ATTN_LONG_FROM")) c->attn_long_from = std::max(0, atoi(e));
         c->trace = getenv("PASS_TRACE") != nullptr;
         int dev = 0, sms = 0;
