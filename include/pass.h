@@ -370,10 +370,18 @@ int pass_linear_noalloc(pass_ctx *ctx, int which, int layer, const float *x_devi
  *       PASS_ERR_TIMEOUT with the sequence state untouched.
  *   PASS_HOOK_ATTN_STALE, value n >= 0: the attention kernel's early fetch pretends the cache is n
  *       positions shorter than it is, which forces its re-check and restart path.
+ *   PASS_HOOK_ATTN_LONG_FROM, value n >= 0: a step counts as "long" (other attention launch shape; with
+ *       d_head 128 and at most 16 rows per sequence the tcgen05 attention kernel) as soon as one sequence
+ *       has n cached positions.  Default 3072 (PASS_ATTN_LONG_FROM in the environment at creation); 0
+ *       sends every step down the long path, so that small test cases reach it.
+ *   PASS_HOOK_ATTN_STUCK, value 0/1: the tcgen05 attention kernel never announces its scores, so its
+ *       bounded waits run out; the call returns PASS_ERR_TIMEOUT with the sequence state untouched.
  * Errors: INVALID_ARG.
  */
 #define PASS_HOOK_GEMM_STUCK 0
 #define PASS_HOOK_ATTN_STALE 1
+#define PASS_HOOK_ATTN_LONG_FROM 2
+#define PASS_HOOK_ATTN_STUCK 3
 int pass_debug_set(pass_ctx *ctx, int hook, int value);
 
 /* Number of kernel launches (graph nodes) of the last pass_step / pass_step_enqueue. */

@@ -156,7 +156,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
                     umma_bf16(tmem + s * 32, a_desc, b_desc, idesc, kk > 0 ? 1u : 0u);
                 }
                 umma_commit(b_ek + 8 * s);       // the key block may be overwritten
-                umma_commit(b_sf + 8 * s);       // the scores are complete
+                if (!p.debug_stuck) umma_commit(b_sf + 8 * s);       // the scores are complete
             }
         }
     } else {

@@ -159,6 +159,7 @@ struct pass_ctx {
     AttnTcMaps attn_tc_maps;      // the key and the value cache as matrices of 128 columns
     bool attn_cluster = true;     // PASS_ATTN_NO_CLUSTER: merge attention slices through global memory
     int attn_debug_stale = 0;     // pass_debug_set(PASS_HOOK_ATTN_STALE, n): attention's early part works from a cache length n short
+    int attn_test_stuck = 0;      // pass_debug_set(PASS_HOOK_ATTN_STUCK, 1): k_attn_tc never announces its scores
     int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
     // Function attributes and occupancy answers belong to the device the context lives on, so they are
     // remembered per context, never per process.
@@ -696,6 +697,7 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
         ap.out = c->d_attn_bf; ap.lo_row0 = plain ? -1 : rh; ap.debug_stale = c->attn_debug_stale;
         ap.rows_per_block = 0;
         ap.status = c->d_status;
+        ap.debug_stuck = c->attn_test_stuck;
         ap.out_tile_rows = big && !plain ? rh : 0;
         if (M <= 16 && md.dh == kTcDH && c->attn_long && c->attn_tc && c->attn_tc_ready) {
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
@@ -1558,6 +1560,8 @@ int pass_debug_set(pass_ctx* c, int hook, int value) {
     switch (hook) {
         case PASS_HOOK_GEMM_STUCK: c->gemm_test_stuck = value ? 1 : 0; break;
         case PASS_HOOK_ATTN_STALE: c->attn_debug_stale = value; break;
+        case PASS_HOOK_ATTN_LONG_FROM: c->attn_long_from = value; break;
+        case PASS_HOOK_ATTN_STUCK: c->attn_test_stuck = value ? 1 : 0; break;
         default: return PASS_ERR_INVALID_ARG;
     }
     // the hooks are part of the launch parameters, which captured graphs hold by value
