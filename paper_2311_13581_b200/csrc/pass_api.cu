@@ -708,7 +708,6 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
             // Long contexts: the key loop (tensor-core work of 4 warps) outweighs everything that one CTA per
             // SM buys at short contexts, so the slices are doubled - two CTAs per SM, 8 warps on the keys.
             if (c->attn_long && ap.n_split * 2 <= 8) ap.n_split *= 2;
-            if (const char* e = getenv("PASS_ATTN_SPLIT")) ap.n_split = std::max(1, std::min(std::min(kAttnMaxSplit, 2 * kMaxCtas / (md.H * n_seq)), atoi(e)));
             if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
             else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
         } else {
