@@ -294,6 +294,10 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_FOOTPRINT    10  /* int32 [6]: shared memory in bytes of the step's GEMM kernel (static, dynamic at 9..16
                                      rows) and of its attention kernel (static, dynamic), the SM's total and what the
                                      system reserves per block: the two kernels are meant to fit on one SM together */
+#define PASS_DBG_ATTN_TRACE   11  /* uint64 [launch][16][16][8]: stamps of the long-cache attention kernel's launches since
+                                     the last read (PASS_TRACE set, one sequence): per (head / 4, key slice) of every
+                                     fourth head: entry, dependency wait over, first key block in shared memory, last
+                                     score product issued, last softmax done, slice stored, head merged (last slice) */
 int pass_get_debug(pass_ctx *ctx, int what, void *dst, size_t bytes);
 
 /*

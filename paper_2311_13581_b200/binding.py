@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libpass_b200.so")
 PASS_DBG_LOGITS, PASS_DBG_DRAFT_LOGITS, PASS_DBG_KV_LEN, PASS_DBG_N_DRAFT = 0, 1, 2, 3
 PASS_DBG_DRAFTS, PASS_DBG_PENDING, PASS_DBG_N_ACCEPTED, PASS_DBG_STATUS, PASS_DBG_HIDDEN = 4, 5, 6, 7, 8
 PASS_DBG_FOOTPRINT = 10
+PASS_DBG_ATTN_TRACE = 11
 PASS_MAX_ROWS = 128
 PASS_HOOK_GEMM_STUCK, PASS_HOOK_ATTN_STALE, PASS_HOOK_ATTN_LONG_FROM, PASS_HOOK_ATTN_STUCK = 0, 1, 2, 3
 PASS_PROMPT_HI_LO, PASS_PROMPT_BF16 = 0, 1

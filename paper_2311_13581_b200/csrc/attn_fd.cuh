@@ -39,6 +39,7 @@ struct AttnParams {
     int out_tile_rows;             // > 0: output rows are laid out in token tiles of this many rows, hi rows of a tile
                                    // followed by its lo rows (the layout the next GEMM of a prompt chunk reads)
     int* status;                   // kStatusTimeout is raised here (k_attn_tc, the only attention kernel that waits)
+    unsigned long long* trace;     // k_attn_tc, PASS_TRACE: [head / 4][16 slices][8] %globaltimer stamps of every fourth head's CTAs
     int debug_stuck;               // test hook (k_attn_tc): the scores are never announced, so the bounded waits run out
     int rows_per_block;            // 0: blockIdx.y = sequence, M rows each (a decode step).  > 0: ONE sequence of M rows
                                    // (a prompt chunk), blockIdx.y = block of rows_per_block rows - causal flash attention

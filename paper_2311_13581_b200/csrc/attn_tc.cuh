@@ -67,6 +67,11 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// Stamps of every fourth head's CTAs only: reads of %globaltimer from all CTAs at once queue up behind one another.
+// Slots: 0 entry, 1 dependency wait over, 2 first key block in shared memory, 3 last score product issued,
+// 4 last softmax / P V done, 5 slice's partial output in memory, 6 slices of the head merged.
+#define PASS_ATTN_TRACE(slot) do { if (p.trace && (blockIdx.x & 3) == 0) p.trace[((blockIdx.x >> 2) * 16 + blockIdx.z) * 8 + (slot)] = global_ns(); } while (0)
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     // aligned to 1024 bytes by hand below: asking for it here would pad the static shared memory of EVERY kernel
@@ -79,6 +84,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     const int head = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = p.M, row0 = b * M;
+    if (tid == 0) PASS_ATTN_TRACE(0);
     const uint32_t base = (smem_u32(smem_tc) + 1023u) & ~1023u;
     const uint32_t sK = base, sV = sK + 2 * kTcTile, sQ = sV + 2 * kTcTile, sP = sQ + kTcQBytes;
     const uint32_t bar = smem_u32(&s_bar[0]);
@@ -103,6 +109,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     const uint32_t tmem = s_tmem;
     griddep_launch_dependents();
     griddep_wait();                                   // the queries and this step's cache rows come from the kernel before
+    if (tid == 0) PASS_ATTN_TRACE(1);
 
     // this CTA's slice of the keys, in whole blocks
     const int seq = __ldcg(p.row_seq + row0), len = __ldcg(p.row_pos + row0);
@@ -148,6 +155,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
                 const uint32_t par = (j >> 1) & 1;
                 if (!mbar_wait(b_fk + 8 * s, par, &s_abort, p.status)) break;
                 if (!mbar_wait(b_se + 8 * s, par ^ 1, &s_abort, p.status)) break;
+                if (j == 0) PASS_ATTN_TRACE(2);
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kTcDH / 16; kk++) {
@@ -158,6 +166,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
                 umma_commit(b_ek + 8 * s);       // the key block may be overwritten
                 if (!p.debug_stuck) umma_commit(b_sf + 8 * s);       // the scores are complete
             }
+            PASS_ATTN_TRACE(3);
         }
     } else {
         // ---------------------------------------------------------------- softmax and O += P V
@@ -270,6 +279,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
             if (lane == 0) mbar_arrive(b_ev + 8 * s);               // the value block may be overwritten
         }
         (void)t;
+        if (warp == 2 && lane == 0) PASS_ATTN_TRACE(4);
     }
     __syncthreads();
     if (*(volatile int*)&s_abort) {
@@ -337,6 +347,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     __threadfence();
     __syncthreads();
     if (tid == 0) {
+        PASS_ATTN_TRACE(5);
         const int prev = atomicAdd(p.counters + b * p.md.H + head, 1);
         s_last = prev == p.n_split - 1;
         if (s_last) p.counters[b * p.md.H + head] = 0;
@@ -348,6 +359,10 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     float* sm_f = sm_o;                                              // [n_split][32] weight of slice s for row i
     if (p.n_split <= 4) attn_merge<kTcDH, 4, 4, kTcThreads>(p, hb, row0, head, sm_f);
     else attn_merge<kTcDH, kAttnMaxSplit, 2, kTcThreads>(p, hb, row0, head, sm_f);
+    if (p.trace) {
+        __syncthreads();
+        if (tid == 0) PASS_ATTN_TRACE(6);
+    }
 }
 
 }  // namespace pass

@@ -191,7 +191,7 @@ struct pass_ctx {
     bool packed = false;               // the GEMMs stream the packed copy of the weights (PASS_NO_PACK: the caller's matrices)
     char* d_packed = nullptr;
     bool trace = false;                // PASS_TRACE=1: chain launches leave timestamps (see PASS_DBG_TRACE)
-    int trace_launch = 0;
+    int trace_launch = 0, attn_trace_launch = 0;
     int chain_done_total[kMaxOps] = {0, 0, 0, 0};   // host mirror of what the counters reach (see launch_chain)
     int* d_chain_flags = nullptr;      // [kMaxOps] tiles done per GEMM position of a chain, growing until the next clear
     std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd;
@@ -393,10 +393,16 @@ struct ChainOp {
 // The tail of the verify scratch (E, [kMaxRows][V] doubles) doubles as the trace buffer: its rows beyond the
 // first half are only used by steps of more than 64 rows.  nullptr when E is too small for that.
 constexpr int kTraceLaunches = 48;
+constexpr size_t kAttnTraceWords = 2048;     // per k_attn_tc launch: [64 heads / 4][16 slices][8 stamps]
 static unsigned long long* trace_base(pass_ctx* c) {
-    const size_t total = (size_t)kMaxRows * c->md.V, need = (size_t)kTraceLaunches * kMaxOps * kMaxCtas * 8;
+    const size_t total = (size_t)kMaxRows * c->md.V;
+    const size_t need = (size_t)kTraceLaunches * (kMaxOps * kMaxCtas * 8 + kAttnTraceWords);
     if (need > total / 2) return nullptr;
-    return (unsigned long long*)c->vb.E + (total - need);
+    return (unsigned long long*)c->vb.E + (total - (size_t)kTraceLaunches * kMaxOps * kMaxCtas * 8);
+}
+// the long-cache attention kernel's stamps sit in front of the GEMM chain's
+static unsigned long long* attn_trace_base(pass_ctx* c) {
+    return trace_base(c) ? trace_base(c) - (size_t)kTraceLaunches * kAttnTraceWords : nullptr;
 }
 
 // Launch up to kMaxOps dependent GEMMs as ONE kernel (see k_gemm_tc).  GEMM j of the chain gets its own
@@ -512,7 +518,11 @@ static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
 }
 
 // Long caches, d_head 128, at most 16 rows per sequence: scores on tcgen05 (attn_tc.cuh), one CTA per SM.
-static void launch_attn_tc(pass_ctx* c, const AttnParams& ap, int n_seq) {
+static void launch_attn_tc(pass_ctx* c, const AttnParams& ap_in, int n_seq) {
+    AttnParams ap = ap_in;
+    ap.trace = nullptr;
+    if (c->trace && c->attn_trace_launch < kTraceLaunches && attn_trace_base(c) && c->md.H <= 64 && n_seq == 1)
+        ap.trace = attn_trace_base(c) + (size_t)(c->attn_trace_launch++) * kAttnTraceWords;
     if (!c->attn_tc_smem_set) {
         note_err(c, cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem), "k_attn_tc shared memory size");
         c->attn_tc_smem_set = true;
@@ -922,6 +932,10 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     // the hand-over slots of the <=16-row GEMMs are EMPTY (all bits set) whenever no launch is using them
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.ll_ws, 0xFF, kLLRegionBytes * kMaxOps, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
+    // stamps are told from empty slots by being non-zero
+    if (c->trace && attn_trace_base(c) &&
+        cudaMemsetAsync(attn_trace_base(c), 0, (size_t)kTraceLaunches * (kMaxOps * kMaxCtas * 8 + kAttnTraceWords) * 8, c->stream) != cudaSuccess)
+        return fail(PASS_ERR_CUDA);
     std::vector<double> inv(cfg->d_head / 2);
     for (int i = 0; i < cfg->d_head / 2; i++)
         inv[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->d_head);
@@ -1307,6 +1321,13 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         const size_t n = std::min(bytes, (size_t)kTraceLaunches * kMaxOps * kMaxCtas * 8 * 8);
         CUDA_TRY(cudaMemcpy(dst, trace_base(c), n, cudaMemcpyDeviceToHost));
         c->trace_launch = 0;
+        return PASS_OK;
+    }
+    if (what == PASS_DBG_ATTN_TRACE) {
+        if (!attn_trace_base(c)) return PASS_ERR_STATE;
+        const size_t n = std::min(bytes, (size_t)kTraceLaunches * kAttnTraceWords * 8);
+        CUDA_TRY(cudaMemcpy(dst, attn_trace_base(c), n, cudaMemcpyDeviceToHost));
+        c->attn_trace_launch = 0;
         return PASS_OK;
     }
     if (what == PASS_DBG_FOOTPRINT) {
