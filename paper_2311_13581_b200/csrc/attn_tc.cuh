@@ -171,7 +171,7 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
     } else {
         // ---------------------------------------------------------------- softmax and O += P V
         const int sw = warp - 2, wg = sw >> 2, quad = warp & 3;      // a warp reaches TMEM lanes 32 * (warp % 4) ..
-        const int g = lane >> 2, t = lane & 3;
+        const int g = lane >> 2;
         {
             // queries, scaled by log2(e) / sqrt(d_head) so that exp2 can be used, as bf16 hi + lo rows of operand B
             const int st = sw * 32 + lane, r = st >> 4, c = st & 15;
@@ -278,7 +278,6 @@ k_attn_tc(const __grid_constant__ AttnTcMaps maps, const AttnParams p) {
             __syncwarp();
             if (lane == 0) mbar_arrive(b_ev + 8 * s);               // the value block may be overwritten
         }
-        (void)t;
         if (warp == 2 && lane == 0) PASS_ATTN_TRACE(4);
     }
     __syncthreads();
