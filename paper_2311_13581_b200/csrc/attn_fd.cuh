@@ -152,8 +152,9 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
 // the usual flash-attention split for many rows).  HL = queries and probabilities as bf16 hi + lo pairs;
 // without it they are single bf16 values (prompt chunks in plain bf16, half the MMAs).
 // CHUNK = the rows are one sequence's prompt chunk (rows_per_block, out_tile_rows, optional lo parts); the
-// decode step's instances have it off and carry none of that code.
-template <int DH, int MT, bool CL, bool HL = true, bool CHUNK = false>
+// decode step's instances have it off and carry none of that code.  ST = depth of the key / value ring: 3 where the
+// CTA shares its SM with the next GEMM launch's CTA, 2 (64 KB at d_head 128) where three of these CTAs share an SM.
+template <int DH, int MT, bool CL, bool HL = true, bool CHUNK = false, int ST = kAttnStages>
 __global__ void __maxnreg__(168)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
@@ -204,10 +205,10 @@ k_attn_fd(const AttnParams p) {
     // rows of this launch's own chunk ahead of this block are cache rows the awaited kernel writes: in chunk
     // mode only positions before the chunk's first row may be fetched early
     const int early_len = CHUNK ? min(len, *(volatile const int*)(p.row_pos)) : len;
-    const uint32_t sK = smem_u32(smem_attn), sV = sK + kAttnStages * TILE_BYTES;
+    const uint32_t sK = smem_u32(smem_attn), sV = sK + ST * TILE_BYTES;
 
     auto load_block = [&](int blk) {
-        const int st = blk % kAttnStages;
+        const int st = blk % ST;
         const int kb = k_begin + blk * kAttnBK;
         for (int idx = tid; idx < kAttnBK * CH; idx += 128) {
             const int key = idx / CH, c = idx % CH;
@@ -223,7 +224,7 @@ k_attn_fd(const AttnParams p) {
     // first ring fill: blocks of old rows now, the rest (and the queries) after the wait
     uint32_t early = 0;
 #pragma unroll
-    for (int st = 0; st < kAttnStages; st++) {
+    for (int st = 0; st < ST; st++) {
         if (st < nb && min(k_end, k_begin + (st + 1) * kAttnBK) <= early_len) { load_block(st); early |= 1u << st; }
     }
     cp_async_commit();
@@ -239,7 +240,7 @@ k_attn_fd(const AttnParams p) {
         }
     }
 #pragma unroll
-    for (int st = 0; st < kAttnStages; st++) {
+    for (int st = 0; st < ST; st++) {
         if (st < nb && !((early >> st) & 1u)) load_block(st);
         cp_async_commit();
     }
@@ -279,12 +280,12 @@ k_attn_fd(const AttnParams p) {
         if (blk > 0) {
             // everybody is done with block blk-1: its stage takes block blk-1+stages
             __syncthreads();
-            if (blk - 1 + kAttnStages < nb) load_block(blk - 1 + kAttnStages);
+            if (blk - 1 + ST < nb) load_block(blk - 1 + ST);
             cp_async_commit();
         }
-        cp_async_wait<kAttnStages - 1>();
+        cp_async_wait<ST - 1>();
         __syncthreads();
-        const int st = blk % kAttnStages;
+        const int st = blk % ST;
         const uint32_t kS = sK + st * TILE_BYTES, vS = sV + st * TILE_BYTES;
 #pragma unroll
         for (int sub = 0; sub < MT; sub++) {

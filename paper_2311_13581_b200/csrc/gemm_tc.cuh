@@ -201,6 +201,18 @@ __device__ __forceinline__ void tmem_ld_wait() {
 __device__ __forceinline__ void epi_bar() {            // the 128 epilogue threads only
     asm volatile("bar.sync 1, 128;" ::: "memory");
 }
+// MANY: kEpiGroups groups of 128 epilogue threads (barriers 1 .. kEpiGroups), and one more barrier for all of them
+constexpr int kEpiGroups = 3;
+template <bool MANY>
+__device__ __forceinline__ void epi_bar_g(int group) {
+    if (!MANY) asm volatile("bar.sync 1, 128;" ::: "memory");
+    else asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+}
+template <bool MANY>
+__device__ __forceinline__ void epi_bar_all() {
+    if (!MANY) asm volatile("bar.sync 1, 128;" ::: "memory");
+    else asm volatile("bar.sync %0, %1;" ::"n"(kEpiGroups + 1), "n"(kEpiGroups * 128) : "memory");
+}
 
 // Shared-memory matrix descriptor: K-major tile with 128-byte rows, 128B swizzle; 8-row groups are
 // 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100).
@@ -304,6 +316,7 @@ struct EpiCtx {
     const unsigned long long* s_kvoff;   // [kTokTile] cache offset of head 0, feature 0 of each token row (kEpiQKV)
     int row_base;            // first token row of the token tile being finished (0 unless the rows are tiled)
     int rows_live;           // live rows of that token tile; s_rstd / s_kvoff are indexed by the row within the tile
+    int group;               // epilogue group of this thread (0 unless the kernel has two)
     int out_row_base;        // row of xn_out / act_out that holds the tile's first token (its lo part xn_lo_row0 further
                              // down): token tiles of hi | lo rows are laid out one after another, as the next GEMM reads them
 };
@@ -317,7 +330,7 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 // loaded (so that this trip to L2 overlaps with another); nullptr = load them here.
 // g_pre / cs_pre: likewise the next norm's gain for this feature (kEpiResid) and the eight rotation pairs
 // (kEpiQKV), fetched by the caller while it was still waiting for the accumulator.
-template <int NR, bool BIG>
+template <int NR, bool BIG, bool MANY = false>
 __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec, int tile, int c0, float (&v)[NR],
                                           const float* hv_pre = nullptr, const float* g_pre = nullptr,
                                           const float2* cs_pre = nullptr) {
@@ -393,12 +406,12 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
 #pragma unroll
             for (int j = 0; j < NR; j++) ss[j] += __shfl_xor_sync(0xffffffffu, ss[j], o);
         }
-        epi_bar();                                  // s_x free
+        epi_bar_g<MANY>(ec.group);                                  // s_x free
         if (lane == 0) {
 #pragma unroll
             for (int j = 0; j < NR; j++) ec.s_x[warp_q * NR + j] = ss[j];
         }
-        epi_bar();
+        epi_bar_g<MANY>(ec.group);
         if (L < NR && c0 + L < rows_live)
             p.sumsq_out[(size_t)tile * kRowsCap + row_base + c0 + L] =
                 ec.s_x[L] + ec.s_x[NR + L] + ec.s_x[2 * NR + L] + ec.s_x[3 * NR + L];
@@ -406,10 +419,10 @@ __device__ __forceinline__ void epi_store(const GemmParams& p, const EpiCtx& ec,
         // Both halves of the threads work after the exchange: a gate lane finishes the even rows of its
         // feature (it reads the up values from the exchange buffer), the matching up lane the odd rows
         // (it reads the gate values).
-        epi_bar();                                  // s_x free
+        epi_bar_g<MANY>(ec.group);                                  // s_x free
 #pragma unroll
         for (int j = 0; j < NR; j++) ec.s_x[L * 9 + j] = v[j];
-        epi_bar();
+        epi_bar_g<MANY>(ec.group);
         const int feat = L & 63, other = L < 64 ? L + 64 : L - 64, n = tile * 64 + feat;
         if (n < p.n_out) {
 #pragma unroll
@@ -573,7 +586,7 @@ __device__ __forceinline__ void weight_xy(const GemmParams& p, int y_rowmajor, i
 // BIG = false: the decode step's kernel (hi | lo rows, one token tile).  BIG = true adds what prompt chunks
 // need (token tiles, plain bf16 rows, whole-unit schedule, loads one row group ahead in the epilogue); it is a
 // second instantiation so that the step's kernel keeps its registers.
-template <bool BIG>
+template <bool BIG, bool MANY = false>
 __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const ChainParams& cp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
@@ -587,7 +600,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
     // 512 bytes more and the two no longer fit side by side)
     __shared__ float s_rstd[BIG ? kTokTile : kMaxRows];
     __shared__ unsigned long long s_kvoff[BIG ? kTokTile : kMaxRows];
-    __shared__ float s_x[128 * 9];
+    __shared__ float s_x[(MANY ? kEpiGroups : 1) * 128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
     constexpr int kPieceCache = 16;
@@ -622,7 +635,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; s++) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, 4); }
+        for (int b = 0; b < 2; b++) { mbar_init(bar_accf + 8 * b, 1); mbar_init(bar_acce + 8 * b, MANY ? 4 * kEpiGroups : 4); }
         s_abort = 0;
         s_issued = 0;
         s_issued_b = 0;
@@ -753,15 +766,18 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                 PASS_TRACE(oi, 2);
             }
         }
-    } else if (warp >= 2 && warp <= 5) {
-        // ---------------------------------------------------------------- epilogue (128 threads)
+    } else if ((warp >= 2 && warp <= 5) || (MANY && warp >= 8)) {
+        // ---------------------------------------------------------------- epilogue (128 threads; MANY: kEpiGroups
+        // groups of 128, warps 2-5, 8-11, 12-15, which share every tile: the passes of eight token rows go round)
         const int wq = warp & 3;                      // TMEM lanes 32*wq .. 32*wq+31
+        const int ge = MANY && warp >= 8 ? (warp - 4) >> 2 : 0;
         EpiCtx ec;
         ec.lane_in_tile = wq * 32 + lane;
         ec.s_rstd = s_rstd;
-        ec.s_x = s_x;
+        ec.s_x = s_x + ge * 128 * 9;
         ec.s_kvoff = s_kvoff;
-        const int et = (warp - 2) * 32 + lane;        // 0..127
+        ec.group = ge;
+        const int et = (warp - (ge ? 4 + 4 * ge : 2)) * 32 + lane;        // 0..127 within the group
         griddep_wait();
         int pidx = 0;
         bool ok = true;
@@ -770,9 +786,9 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
             const GemmParams& p = cp.op[oi];
             if (oi > 0) {
                 // one thread waits for the previous GEMM; the outcome is made uniform through the barrier
-                if (et == 0 && !wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status))
+                if (et == 0 && ge == 0 && !wait_count(cp.op_done + oi - 1, cp.op_target[oi - 1], &s_abort, cp.status))
                     *(volatile int*)&s_epi_fail = 1;
-                epi_bar();
+                epi_bar_all<MANY>();                 // (both groups leave together, and nobody still reads the row tables)
                 if (*(volatile int*)&s_epi_fail) { ok = false; break; }
             }
             // rstd of the input rows: eight lanes per row, each sums every eighth part (its loads are
@@ -809,7 +825,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
             ec.out_row_base = 0;
             ec.rows_live = p.R;
             if (!BIG || p.n_tok_tiles == 0) fill_row_tables(0, p.R);
-            epi_bar();
+            epi_bar_g<MANY>(ge);
             const bool has_lo = !BIG || p.has_lo;
             const int rows_acc = has_lo ? p.rh : p.npad;            // token rows held by an accumulator
             const size_t slot_floats = (size_t)rows_acc * kTileN;
@@ -820,7 +836,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
                 float2 cs_pre[16] = {};
-                const bool pre = p.rh == 16 && has_lo && pc.index == 0;
+                const bool pre = !MANY && p.rh == 16 && has_lo && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
@@ -836,7 +852,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     ftile = pc.tile / p.n_tok_tiles;
                     const int tt = pc.tile % p.n_tok_tiles;
                     if (tt != cur_tt) {                        // another token tile: its rows' factors and cache offsets
-                        epi_bar();
+                        epi_bar_g<MANY>(ge);
                         const int tile_tokens = p.has_lo ? p.rh : p.npad;
                         ec.row_base = tt * tile_tokens;
                         ec.out_row_base = tt * p.npad;
@@ -847,12 +863,12 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                 }
                 // each thread waits for itself; the outcome is made uniform before any barrier is used
                 if (!mbar_wait(bar_accf + 8 * buf, (pidx >> 1) & 1, &s_abort, cp.status)) *(volatile int*)&s_epi_fail = 1;
-                epi_bar();
+                epi_bar_all<MANY>();
                 if (*(volatile int*)&s_epi_fail) { ok = false; break; }
-                if (et == 0) PASS_TRACE(oi, 4);
+                if (et == 0 && ge == 0) PASS_TRACE(oi, 4);
                 tc_fence_after();
                 const bool whole = pc.n_pieces == 1;
-                const bool ll = p.rh == 16 && has_lo;          // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
+                const bool ll = !MANY && p.rh == 16 && has_lo;          // 9..16 rows (padded to 16): counter-free hand-over, fixed finisher
                 float* ll_peer = nullptr;                      // finisher: the slots to mark empty once the tile is out
                 int ll_n = 0;
                 const uint32_t t_addr = tmem_base + ((uint32_t)(wq * 32) << 16) + buf * cp.npad;
@@ -907,66 +923,59 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                             if (!whole)
                                 ll_gather<kLLRows>(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
                             if (et == 0 && c0 == 0 && !whole) PASS_TRACE(oi, 5);
-                            epi_store<kLLRows, BIG>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
+                            epi_store<kLLRows, BIG, MANY>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
                                                p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs9 : nullptr);
                         }
                         if (!whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
                     }
-                } else if (!BIG && has_lo) {
-                    // More than 16 token rows (k = 8, batches): the same counter-free hand-over, sixteen rows at a
-                    // time, each group as two passes of eight rows through the epilogue.
+                } else if (MANY) {
+                    // More than 16 token rows (k = 8, batches): the same counter-free hand-over, eight rows at a time;
+                    // pass q (rows 8q .. 8q+7) belongs to epilogue group q mod kEpiGroups.
                     const bool contributor = !whole && pc.index != 0;
                     float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
                     const size_t peer_stride = 2 * slot_floats;
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
                     if (p.epi == kEpiResid) g_pre = n < p.n_out ? __bfloat162float(p.gain_next[n]) : 0.f;
                     if (!contributor) tile_done = true;
+                    const int n_pass = p.rh / 8;
+                    bool released = false;
+                    auto release_acc = [&]() {              // this warp has read the accumulator out: the MMA warp may have it back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
+                        released = true;
+                    };
 #pragma unroll 1
-                    for (int rg = 0; rg < p.rh; rg += 16) {
-                        float av[16];
-#pragma unroll
-                        for (int c0 = 0; c0 < 16; c0 += 8) {
+                    for (int q = ge; q < n_pass; q += kEpiGroups) {
+                        const int row = 8 * q;
+                        float a8[8];
+                        {
                             float hi[8], lo[8];
-                            if (rg + c0 < p.rh) {
-                                tmem_ld8(t_addr + rg + c0, hi);
-                                tmem_ld8(t_addr + p.rh + rg + c0, lo);
-                                tmem_ld_wait();
-                            }
+                            tmem_ld8(t_addr + row, hi);
+                            tmem_ld8(t_addr + p.rh + row, lo);
+                            tmem_ld_wait();
 #pragma unroll
-                            for (int j = 0; j < 8; j++) av[c0 + j] = rg + c0 < p.rh ? hi[j] + lo[j] : 0.f;
+                            for (int j = 0; j < 8; j++) a8[j] = hi[j] + lo[j];
                         }
-                        if (rg + 16 >= p.rh) {              // the accumulator has been read out: the MMA warp may have it back
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
-                        }
-                        if (rg >= p.R) continue;
+                        if (q + kEpiGroups >= n_pass) release_acc();
+                        if (row >= p.R) continue;
                         if (contributor) {
                             float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
 #pragma unroll
-                            for (int j = 0; j < 16; j++)
-                                if (rg + j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)(rg + j) * kTileN, __float_as_uint(av[j]));
+                            for (int j = 0; j < 8; j++)
+                                if (row + j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)(row + j) * kTileN, __float_as_uint(a8[j]));
                             continue;
                         }
-                        float hv[16];
+                        float h8[8];
 #pragma unroll
-                        for (int j = 0; j < 16; j++)
-                            hv[j] = (p.epi == kEpiResid && rg + j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)(rg + j) * p.n_out + n) : 0.f;
-#pragma unroll 1
-                        for (int c0 = 0; c0 < 16; c0 += 8) {
-                            if (rg + c0 >= p.R) break;
-                            float a8[8], h8[8];
-#pragma unroll
-                            for (int j = 0; j < 8; j++) {
-                                a8[j] = c0 == 0 ? av[j] : av[8 + j];
-                                h8[j] = c0 == 0 ? hv[j] : hv[8 + j];
-                            }
-                            if (!whole)
-                                ll_gather<8>(peer, peer_stride, pc.n_pieces - 1, rg + c0, min(p.R - rg - c0, 8), a8, &s_abort, cp.status);
-                            epi_store<8, BIG>(p, ec, pc.tile, rg + c0, a8, p.epi == kEpiResid ? h8 : nullptr,
-                                              p.epi == kEpiResid ? &g_pre : nullptr, nullptr);
-                        }
+                        for (int j = 0; j < 8; j++)
+                            h8[j] = (p.epi == kEpiResid && row + j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)(row + j) * p.n_out + n) : 0.f;
+                        if (!whole)
+                            ll_gather<8>(peer, peer_stride, pc.n_pieces - 1, row, min(p.R - row, 8), a8, &s_abort, cp.status);
+                        epi_store<8, BIG, MANY>(p, ec, pc.tile, row, a8, p.epi == kEpiResid ? h8 : nullptr,
+                                                p.epi == kEpiResid ? &g_pre : nullptr, nullptr);
                     }
+                    if (!released) release_acc();
                     if (!contributor && !whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
                 } else if (BIG) {               // prompt chunks (the step's kernel never gets here: it has hi | lo rows)
                 float* my_slot = p.partial_ws + ((size_t)cta * 2 + pc.slot) * slot_floats;
@@ -997,7 +1006,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         for (int j = 0; j < 8; j++) hi[j] += lo[j];
                     }
                     if (whole) {
-                        epi_store<8, BIG>(p, ec, ftile, c0, hi, ahead ? hv_cur : nullptr, ahead ? &g_res : nullptr);
+                        epi_store<8, BIG, MANY>(p, ec, ftile, c0, hi, ahead ? hv_cur : nullptr, ahead ? &g_res : nullptr);
                         if (ahead) {
 #pragma unroll
                             for (int j = 0; j < 8; j++) hv_cur[j] = hv_nxt[j];
@@ -1018,7 +1027,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     // parts in k order.  The barrier orders every thread's partial stores before thread 0's
                     // acq_rel atomic (release is cumulative), and the loads after the second barrier behind
                     // its acquire.
-                    epi_bar();
+                    epi_bar_g<MANY>(ge);
                     if (et == 0) {
                         if (cp.test_stuck && oi == 0 && pc.index != 0) {
                             s_last = 0;             // test hook: this part is never announced, the tile never finishes
@@ -1030,7 +1039,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                             if (s_last) p.tile_counters[pc.tile] = 0;
                         }
                     }
-                    epi_bar();
+                    epi_bar_g<MANY>(ge);
                     if (et == 0) PASS_TRACE(oi, 5);
                     if (s_last) {
                         tile_done = true;
@@ -1063,23 +1072,24 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                                     }
                                 }
                             }
-                            epi_store<8, BIG>(p, ec, pc.tile, c0, acc);
+                            epi_store<8, BIG, MANY>(p, ec, pc.tile, c0, acc);
                         }
                     }
                 }
                 }
-                if (et == 0 && tile_done && !whole) PASS_TRACE(oi, 6);
-                if (signal && tile_done) {
-                    // every thread's stores of this tile happen-before thread 0's release (barrier + cumulativity)
-                    epi_bar();
-                    if (et == 0)
+                if (et == 0 && ge == 0 && tile_done && !whole) PASS_TRACE(oi, 6);
+                if ((signal || MANY) && tile_done) {
+                    // every thread's stores of this tile happen-before thread 0's release (barrier + cumulativity);
+                    // with two groups the barrier also keeps the reset below behind the other group's reads
+                    epi_bar_all<MANY>();
+                    if (signal && et == 0 && ge == 0)
                         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cp.op_done + oi) : "memory");
-                    if (et == 0) PASS_TRACE(oi, 7);
+                    if (et == 0 && ge == 0) PASS_TRACE(oi, 7);
                 }
-                if (ll_peer) ll_reset(ll_peer, 2 * slot_floats, ll_n, p.R);
+                if (ll_peer && ge == 0) ll_reset(ll_peer, 2 * slot_floats, ll_n, p.R);
             }
-            if (et == 0) *(volatile int*)&s_epi_done = oi;
-            if (et == 0) PASS_TRACE(oi, 3);
+            if (et == 0 && ge == 0) *(volatile int*)&s_epi_done = oi;
+            if (et == 0 && ge == 0) PASS_TRACE(oi, 3);
         }
     }
 
@@ -1106,6 +1116,14 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
 __global__ void __maxnreg__(168)
 k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
     gemm_chain_body<false>(maps, cp);
+}
+// Steps of more than 16 token rows (k = 8, batches): the many-row epilogue in place of the 16-row one, run by
+// kEpiGroups groups of four warps (512 threads: the attention CTA no longer fits beside this one, which at these
+// row counts costs less than the extra groups save).
+constexpr int kGemmThreadsMany = 128 + kEpiGroups * 128;
+__global__ void __launch_bounds__(kGemmThreadsMany, 1)
+k_gemm_tc_many(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    gemm_chain_body<false, true>(maps, cp);
 }
 // prompt chunks: alone on its SM (192 KB of ring), so the register cap of the step's kernel does not apply
 __global__ void __launch_bounds__(kGemmThreads, 1)

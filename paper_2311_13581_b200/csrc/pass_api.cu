@@ -163,7 +163,7 @@ struct pass_ctx {
     int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
     // Function attributes and occupancy answers belong to the device the context lives on, so they are
     // remembered per context, never per process.
-    size_t gemm_smem_set = 0, gemm_big_smem_set = 0;
+    size_t gemm_smem_set = 0, gemm_big_smem_set = 0, gemm_many_smem_set = 0;
     std::map<int, bool> attn_attr_set;         // by kernel instance
     std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
@@ -337,6 +337,10 @@ static bool make_map_packed(CUtensorMap* m, const void* base, uint64_t n_boxes, 
 // Token rows are padded to a multiple of 8 per half (hi | lo).  Up to 16 rows always take 16 per half: that is
 // the padding with the counter-free hand-over of partial sums (see k_gemm_tc), and a one-row step is then as
 // fast as a nine-row one (3.10 -> 3.06 ms at the 7B shape) for 2 KB more activation bytes per stage.
+// From this many token rows on a step's GEMMs run in k_gemm_tc_many: the passes of eight rows through the epilogue
+// are shared by three groups of warps, which beats the nine-row passes of one group from two passes on (k >= 5:
+// 3.55 -> 3.46 ms at 13 rows) although the attention CTA no longer fits beside the GEMM CTA.
+constexpr int kManyRowsFrom = 10;
 static int npad_for(int R) { return R <= 16 ? 32 : ((2 * R + 15) / 16) * 16; }
 
 static int gemm_stages(int npad) {
@@ -441,8 +445,9 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
         for (int q = 0; q < 4; q++) maps.m[j][q] = ops[0].a0;
     const size_t smem = (size_t)cp.stages * (kATileBytes + cp.npad * 128) + 1024;
     const bool big = ops[0].p.whole_only != 0;        // a prompt chunk: the kernel instance with token tiles
-    auto kern = big ? k_gemm_tc_big : k_gemm_tc;
-    size_t& smem_set = big ? c->gemm_big_smem_set : c->gemm_smem_set;
+    const bool many = !big && ops[0].p.R >= kManyRowsFrom;        // the instance with several epilogue groups
+    auto kern = big ? k_gemm_tc_big : many ? k_gemm_tc_many : k_gemm_tc;
+    size_t& smem_set = big ? c->gemm_big_smem_set : many ? c->gemm_many_smem_set : c->gemm_smem_set;
     if (smem > smem_set) {
         note_err(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "k_gemm_tc shared memory size");
         // all of the SM's L1/shared storage as shared memory: lets the CTA of the next launch become
@@ -456,7 +461,7 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     for (int j = 0; j < n_ops; j++) units = std::max(units, (long long)ops[j].p.n_tiles * ops[j].p.kb_per_tile);
     // a chain needs every CTA resident at once (they wait for one another's tiles): one CTA per SM
     cfg.gridDim = dim3((unsigned)std::min<long long>(c->n_sms, units));
-    cfg.blockDim = dim3(kGemmThreads);
+    cfg.blockDim = dim3(many ? kGemmThreadsMany : kGemmThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = c->stream;
     cudaLaunchAttribute at[1];
@@ -484,13 +489,13 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
 
 // The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
 // attention, O GEMM (+residual, next norm's input), gate/up GEMM (+SwiGLU), down GEMM (+residual).
-template <int DH, int MT, bool CL>
+template <int DH, int MT, bool CL, int ST>
 static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
-    constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
-    bool& set = c->attn_attr_set[DH * 8 + MT * 2 + (CL ? 1 : 0)];
+    constexpr int smem = 2 * ST * kAttnBK * DH * 2;
+    bool& set = c->attn_attr_set[ST * 4096 + DH * 8 + MT * 2 + (CL ? 1 : 0)];
     if (!set) {
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_attn_fd carveout");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST>, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_attn_fd carveout");
         set = true;
     }
     cudaLaunchConfig_t cfg;
@@ -513,7 +518,7 @@ static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     }
     cfg.attrs = at;
     cfg.numAttrs = na;
-    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL>, ap), "k_attn_fd launch");
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL, true, false, ST>, ap), "k_attn_fd launch");
     c->launches++;
 }
 
@@ -545,14 +550,14 @@ static void launch_attn_tc(pass_ctx* c, const AttnParams& ap_in, int n_seq) {
 // Can the slices of every (sequence, head) run as one cluster each, all at the same time?  Asked once per
 // context, kernel instance, slice count and batch; if not (or with more than 8 slices) the merge goes through
 // global memory.
-template <int DH, int MT>
+template <int DH, int MT, int ST>
 static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
     if (!c->attn_cluster || n_split < 2 || n_split > 8) return false;
-    const int key = ((DH * 8 + MT) * 32 + n_split) * 256 + n_seq;
+    const int key = (((ST * 256 + DH) * 8 + MT) * 32 + n_split) * 256 + n_seq;
     auto it = c->attn_cluster_max.find(key);
     if (it == c->attn_cluster_max.end()) {
-        constexpr int smem = 2 * kAttnStages * kAttnBK * DH * 2;
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        constexpr int smem = 2 * ST * kAttnBK * DH * 2;
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, true, true, false, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
         cfg.gridDim = dim3(c->md.H, n_seq, n_split);
@@ -564,16 +569,16 @@ static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
         cfg.attrs = at;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true, true, false, ST>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
         it = c->attn_cluster_max.emplace(key, n).first;
     }
     return it->second >= c->md.H * n_seq;
 }
 
-template <int DH, int MT>
+template <int DH, int MT, int ST = kAttnStages>
 static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
-    if (attn_cluster_ok<DH, MT>(c, ap.n_split, n_seq)) launch_attn_fd_impl<DH, MT, true>(c, ap, n_seq);
-    else launch_attn_fd_impl<DH, MT, false>(c, ap, n_seq);
+    if (attn_cluster_ok<DH, MT, ST>(c, ap.n_split, n_seq)) launch_attn_fd_impl<DH, MT, true, ST>(c, ap, n_seq);
+    else launch_attn_fd_impl<DH, MT, false, ST>(c, ap, n_seq);
 }
 
 // GEMMs of the decoder layers as chain entries.
@@ -712,6 +717,15 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
         if (M <= 16 && md.dh == kTcDH && c->attn_long && c->attn_tc && c->attn_tc_ready) {
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             launch_attn_tc(c, ap, n_seq);
+        } else if (M <= 32 && R >= kManyRowsFrom) {
+            // A step of ten rows or more: its GEMM kernel (k_gemm_tc_many) leaves no room for an attention CTA on its
+            // SM, so the attention kernel has the SMs to itself: a ring of two stages (64 KB at d_head 128), three
+            // CTAs per SM, and as many slices per (sequence, head) pair as fill those (at most 8, a cluster's worth).
+            const int pairs = md.H * n_seq;
+            ap.n_split = std::max(1, std::min(8, 3 * c->n_sms / pairs));
+            ap.n_split = std::min(ap.n_split, (2 * kMaxCtas + pairs) / pairs);      // what the slices' workspace holds
+            if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1, 2>(c, ap, n_seq); else launch_attn_fd<128, 2, 2>(c, ap, n_seq); }
+            else              { if (M <= 16) launch_attn_fd<64, 1, 2>(c, ap, n_seq); else launch_attn_fd<64, 2, 2>(c, ap, n_seq); }
         } else if (M <= 32) {
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));

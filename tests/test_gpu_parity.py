@@ -280,7 +280,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     shape = SEVENB_2L
     w = si.make_weights(shape, seed=0, device="cuda:0")
     w_cpu = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in w.items()}
-    ctx_len, cap = 512, 600
+    ctx_len, cap = 512, 700
     ctx = pb.PassContext(shape, w, 1, cap)
     be = po.TransformerBackend(shape, w_cpu, cap)
     _load_synthetic_cache(ctx, [be], shape, ctx_len)
@@ -309,6 +309,16 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     stats, _ = lockstep(ctx, [orc], 1, 0.0, 3, step0=6)
     assert stats["max_logit_err"] <= 1e-2, stats
     stats, _ = lockstep(ctx, [orc], 4, 0.0, 2, step0=9)
+    assert stats["max_logit_err"] <= 1e-2, stats
+    # and with 17 rows (k = 8): the many-row instance of the GEMM kernel, whose epilogue groups must all leave
+    # together when one of them gives up
+    stats, _ = lockstep(ctx, [orc], 8, 0.0, 2, step0=11)
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 1)
+    with pytest.raises(pb.PassError) as e:
+        ctx.step(8, 0.0, None)
+    assert "timed out" in str(e.value)
+    ctx.debug_set(pb.PASS_HOOK_GEMM_STUCK, 0)
+    stats, _ = lockstep(ctx, [orc], 8, 0.0, 2, step0=13)
     assert stats["max_logit_err"] <= 1e-2, stats
     ctx.close()
 
