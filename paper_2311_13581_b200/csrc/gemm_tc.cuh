@@ -17,12 +17,13 @@
 //     on whole tiles (see get_piece).  A tile cut across CTAs is summed in k order - deterministic -
 //     by one CTA, which then runs the fused epilogue: the CTA holding the tile's first k-blocks (that
 //     piece is the last of its own range), which finds the other parts in EMPTY-or-value words (no
-//     counter, see ll_gather).  Up to 16 token rows go through that in one or two passes of nine rows;
-//     more rows (k = 8, batches) sixteen at a time.  (The prompt-chunk instantiation computes every unit
+//     counter, see ll_gather).  Up to nine token rows (k <= 4) go through that in one pass of nine rows; more
+//     rows (k >= 5, batches) in passes of eight, in an instantiation of the kernel with three epilogue groups
+//     that take the passes in turn (k_gemm_tc_many).  (The prompt-chunk instantiation computes every unit
 //     whole and shares nothing.)
 //   * warp roles: warp 0 weight loads, warp 6 activation loads, warp 1 TMEM allocation + MMA issue,
-//     warps 2-5 epilogue (TMEM -> registers -> fused epilogue); two accumulator buffers so the epilogue
-//     of one piece overlaps the main loop of the next.
+//     warps 2-5 epilogue (TMEM -> registers -> fused epilogue; k_gemm_tc_many: also warps 8-11 and 12-15);
+//     two accumulator buffers so the epilogue of one piece overlaps the main loop of the next.
 //   * one launch runs a chain of dependent GEMMs (see k_gemm_tc) so that the weight ring never drains
 //     at a GEMM boundary.
 //   * programmatic dependent launch: weight tiles do not depend on the previous kernel, so they are
