@@ -836,7 +836,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                 // what the epilogue of this tile reads besides the accumulator is requested now, so that
                 // the trip to L2 is over by the time the accumulator is complete
                 float g_pre = 0.f;
-                float2 cs_pre[16] = {};
+                float2 cs_pre[kLLRows] = {};
                 const bool pre = !MANY && p.rh == 16 && has_lo && pc.index == 0;
                 if (pre && p.epi == kEpiResid) {
                     const int n = pc.tile * kTileN + ec.lane_in_tile;
@@ -845,7 +845,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                 if (pre && p.epi == kEpiQKV) {
                     const int i2 = ((pc.tile * kTileN + ec.lane_in_tile) % p.md.dh) >> 1;
 #pragma unroll
-                    for (int j = 0; j < 16; j++)
+                    for (int j = 0; j < kLLRows; j++)
                         cs_pre[j] = __ldg(p.rope_cs + (size_t)min(j, p.R - 1) * (p.md.dh / 2) + i2);
                 }
                 int ftile = pc.tile;                           // feature tile of this piece
@@ -900,37 +900,30 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         // were either computed at the very start of their CTAs' ranges or finish together with it.
                         tile_done = true;
                         const int n = pc.tile * kTileN + ec.lane_in_tile;
-                        float hv[16];
+                        float hv[kLLRows];
 #pragma unroll
-                        for (int j = 0; j < 16; j++)
+                        for (int j = 0; j < kLLRows; j++)
                             hv[j] = (p.epi == kEpiResid && j < p.R && n < p.n_out) ? __ldcg(p.h + (size_t)j * p.n_out + n) : 0.f;
                         // every contributor but the first keeps its part in slot 0 (its range begins inside the tile)
                         float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
                         const size_t peer_stride = 2 * slot_floats;
-                        // rows go through the epilogue nine at a time (ONE rolled copy of its code): the 1 + 2k rows
-                        // of up to four look-ahead tokens take a single pass
-#pragma unroll 1
-                        for (int c0 = 0; c0 < 16; c0 += kLLRows) {
-                            if (c0 >= p.R) break;
+                        // the (at most nine) rows go through the epilogue in one pass: the 1 + 2k rows of up to four
+                        // look-ahead tokens (steps of more rows run in k_gemm_tc_many)
+                        {
                             float a9[kLLRows], h9[kLLRows];
                             float2 cs9[kLLRows];
 #pragma unroll
-                            for (int j = 0; j < kLLRows; j++) {
-                                // (row 16 and 17 of the second pass do not exist)
-                                a9[j] = c0 == 0 ? av[j] : (j < 16 - kLLRows ? av[kLLRows + j] : 0.f);
-                                h9[j] = c0 == 0 ? hv[j] : (j < 16 - kLLRows ? hv[kLLRows + j] : 0.f);
-                                cs9[j] = c0 == 0 ? cs_pre[j] : (j < 16 - kLLRows ? cs_pre[kLLRows + j] : make_float2(0.f, 0.f));
-                            }
+                            for (int j = 0; j < kLLRows; j++) { a9[j] = av[j]; h9[j] = hv[j]; cs9[j] = cs_pre[j]; }
                             if (!whole)
-                                ll_gather<kLLRows>(peer, peer_stride, pc.n_pieces - 1, c0, min(p.R - c0, kLLRows), a9, &s_abort, cp.status);
-                            if (et == 0 && c0 == 0 && !whole) PASS_TRACE(oi, 5);
-                            epi_store<kLLRows, BIG, MANY>(p, ec, pc.tile, c0, a9, p.epi == kEpiResid ? h9 : nullptr,
+                                ll_gather<kLLRows>(peer, peer_stride, pc.n_pieces - 1, 0, min(p.R, kLLRows), a9, &s_abort, cp.status);
+                            if (et == 0 && !whole) PASS_TRACE(oi, 5);
+                            epi_store<kLLRows, BIG, MANY>(p, ec, pc.tile, 0, a9, p.epi == kEpiResid ? h9 : nullptr,
                                                p.epi == kEpiResid ? &g_pre : nullptr, p.epi == kEpiQKV ? cs9 : nullptr);
                         }
                         if (!whole) { ll_peer = peer; ll_n = pc.n_pieces - 1; }
                     }
                 } else if (MANY) {
-                    // More than 16 token rows (k = 8, batches): the same counter-free hand-over, eight rows at a time;
+                    // Ten token rows or more (k >= 5, batches): the same counter-free hand-over, eight rows at a time;
                     // pass q (rows 8q .. 8q+7) belongs to epilogue group q mod kEpiGroups.
                     const bool contributor = !whole && pc.index != 0;
                     float* peer = p.ll_ws + ((size_t)(cta + 1) * 2) * slot_floats + ec.lane_in_tile;
@@ -1118,7 +1111,7 @@ __global__ void __maxnreg__(168)
 k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
     gemm_chain_body<false>(maps, cp);
 }
-// Steps of more than 16 token rows (k = 8, batches): the many-row epilogue in place of the 16-row one, run by
+// Steps of ten token rows or more (k >= 5, batches): the many-row epilogue in place of the nine-row one, run by
 // kEpiGroups groups of four warps (512 threads: the attention CTA no longer fits beside this one, which at these
 // row counts costs less than the extra groups save).
 constexpr int kGemmThreadsMany = 128 + kEpiGroups * 128;
