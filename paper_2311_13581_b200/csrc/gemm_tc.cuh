@@ -537,7 +537,7 @@ struct ChainParams {
 };
 // Only every 16th CTA leaves stamps: reads of %globaltimer from all CTAs at once queue up behind one another
 // (tens of microseconds for 148 readers) and would stretch the very hand-overs the trace is meant to show.
-#define PASS_TRACE(oi, slot) do { if (cp.trace && (blockIdx.x & 15) == 0) cp.trace[((size_t)(oi) * gridDim.x + blockIdx.x) * 8 + (slot)] = global_ns(); } while (0)
+#define PASS_TRACE(oi, slot) do { if (TRACE && cp.trace && (blockIdx.x & 15) == 0) cp.trace[((size_t)(oi) * gridDim.x + blockIdx.x) * 8 + (slot)] = global_ns(); } while (0)
 
 __device__ __forceinline__ bool wait_count(const int* counter, int target, volatile int* s_abort, int* g_status) {
     const long long t0 = clock64();
@@ -587,7 +587,7 @@ __device__ __forceinline__ void weight_xy(const GemmParams& p, int y_rowmajor, i
 // BIG = false: the decode step's kernel (hi | lo rows, one token tile).  BIG = true adds what prompt chunks
 // need (token tiles, plain bf16 rows, whole-unit schedule, loads one row group ahead in the epilogue); it is a
 // second instantiation so that the step's kernel keeps its registers.
-template <bool BIG, bool MANY = false>
+template <bool BIG, bool MANY = false, bool TRACE = true>
 __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const ChainParams& cp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[2 * 16 + 4];   // full[S], empty[S], acc_full[2], acc_empty[2]
@@ -668,7 +668,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
                 const GemmParams& p = cp.op[oi];
                 const uint32_t a_box_bytes = p.interleave ? kATileBytes / 2 : kATileBytes;
-                if (cp.hold && oi > 0) {
+                if (TRACE && cp.hold && oi > 0) {
                     const long long t0 = clock64();
                     while (*(volatile int*)&s_epi_done < oi - 1) {
                         if (*(volatile int*)&s_abort || clock64() - t0 > kWaitCycles) { ok = false; break; }
@@ -893,7 +893,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
 #pragma unroll
                         for (int j = 0; j < 16; j++)
-                            if (j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
+                            if (j < p.R && !(TRACE && cp.test_stuck && oi == 0)) st_word(dst + (size_t)j * kTileN, __float_as_uint(av[j]));
                     } else {
                         // A whole tile, or the tile's first part.  The first part is this CTA's LAST piece of the
                         // GEMM (its range ends inside the tile), so it is the natural finisher: the other parts
@@ -957,7 +957,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                             float* dst = p.ll_ws + ((size_t)cta * 2 + pc.slot) * slot_floats + ec.lane_in_tile;
 #pragma unroll
                             for (int j = 0; j < 8; j++)
-                                if (row + j < p.R && !(cp.test_stuck && oi == 0)) st_word(dst + (size_t)(row + j) * kTileN, __float_as_uint(a8[j]));
+                                if (row + j < p.R && !(TRACE && cp.test_stuck && oi == 0)) st_word(dst + (size_t)(row + j) * kTileN, __float_as_uint(a8[j]));
                             continue;
                         }
                         float h8[8];
@@ -1023,7 +1023,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     // its acquire.
                     epi_bar_g<MANY>(ge);
                     if (et == 0) {
-                        if (cp.test_stuck && oi == 0 && pc.index != 0) {
+                        if (TRACE && cp.test_stuck && oi == 0 && pc.index != 0) {
                             s_last = 0;             // test hook: this part is never announced, the tile never finishes
                         } else {
                             int prev;
@@ -1109,7 +1109,14 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
 
 __global__ void __maxnreg__(168)
 k_gemm_tc(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
-    gemm_chain_body<false>(maps, cp);
+    gemm_chain_body<false, false, false>(maps, cp);
+}
+// the same with the %globaltimer stamps, the test hook that withholds partial sums and the held-back weight
+// requests compiled in (template flag TRACE): kept out of the kernel above, whose step time follows its code
+// size (3.00 -> 2.94 ms per nine-row step without the stamps alone)
+__global__ void __maxnreg__(168)
+k_gemm_tc_traced(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    gemm_chain_body<false, false, true>(maps, cp);
 }
 // Steps of ten token rows or more (k >= 5, batches): the many-row epilogue in place of the nine-row one, run by
 // kEpiGroups groups of four warps (512 threads: the attention CTA no longer fits beside this one, which at these
