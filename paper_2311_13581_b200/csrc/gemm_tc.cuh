@@ -662,7 +662,8 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
         // ---------------------------------------------------------------- weight producer
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();
-            int fill = 0;
+            int fill = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             Piece pc;
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
@@ -680,24 +681,26 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     int y;
                     weight_box(p, maps.m[oi], (BIG && p.n_tok_tiles > 0) ? pc.tile / p.n_tok_tiles : pc.tile, 0, m, y);
                     for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                        const int s = fill % S;
-                        const uint32_t parity = ((fill / S) & 1) ^ 1;
-                        if (!mbar_wait(bar_empty + 8 * s, parity, &s_abort, cp.status)) { ok = false; break; }
+                        // (stage and phase are counted along: a division by the ring depth per stage is time this
+                        // single thread does not have)
+                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, &s_abort, cp.status)) { ok = false; break; }
                         mbar_expect_tx(bar_full + 8 * s, a_box_bytes);
                         int wx, wy;
                         weight_xy(p, y, kb, wx, wy);
                         tma_load_2d(tiles_base + s * stage_bytes, m, bar_full + 8 * s, wx, wy, pol_w);
                         fill++;
-                        *(volatile int*)&s_issued = fill;
+                        if (++s == S) { s = 0; ph ^= 1; }
                     }
                 }
             }
+            *(volatile int*)&s_issued = fill;          // for the teardown after a wait that ran out
         }
     } else if (warp == 6) {
         // ---------------------------------------------------------------- activation producer
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-            int fill = 0;
+            int fill = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             Piece pc;
             griddep_wait();                    // the first GEMM's activations are the previous kernel's output
@@ -716,8 +719,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     weight_box(p, maps.m[oi], (BIG && p.n_tok_tiles > 0) ? pc.tile / p.n_tok_tiles : pc.tile, 1, m, y);
                     const int b_row0 = (BIG && p.n_tok_tiles > 0) ? (pc.tile % p.n_tok_tiles) * p.npad : 0;    // token tile
                     for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                        const int s = fill % S;
-                        if (!mbar_wait(bar_empty + 8 * s, ((fill / S) & 1) ^ 1, &s_abort, cp.status)) { ok = false; break; }
+                        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, &s_abort, cp.status)) { ok = false; break; }
                         const uint32_t dst = tiles_base + s * stage_bytes;
                         if (p.interleave) {
                             mbar_expect_tx(bar_full + 8 * s, stage_bytes - a_box_bytes);
@@ -729,16 +731,18 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         }
                         tma_load_2d(dst + kATileBytes, &maps.m[oi][3], bar_full + 8 * s, kb * kBlockK, b_row0, pol_x);
                         fill++;
-                        *(volatile int*)&s_issued_b = fill;
+                        if (++s == S) { s = 0; ph ^= 1; }
                     }
                 }
             }
+            *(volatile int*)&s_issued_b = fill;        // for the teardown after a wait that ran out
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issue
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(cp.npad);
-            int fill = 0, pidx = 0;
+            int pidx = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             Piece pc;
             for (int oi = 0; ok && oi < cp.n_ops; oi++) {
@@ -750,8 +754,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * cp.npad;
                     for (int kb = pc.kb0; kb < pc.kb1; kb++) {
-                        const int s = fill % S;
-                        if (!mbar_wait(bar_full + 8 * s, (fill / S) & 1, &s_abort, cp.status)) { ok = false; break; }
+                        if (!mbar_wait(bar_full + 8 * s, ph, &s_abort, cp.status)) { ok = false; break; }
                         if (first) { PASS_TRACE(oi, 1); first = false; }
                         tc_fence_after();
                         const uint32_t a_addr = tiles_base + s * stage_bytes, b_addr = a_addr + kATileBytes;
@@ -760,7 +763,7 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
                         for (int kk = 0; kk < kBlockK / 16; kk++)
                             umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb > pc.kb0 || kk > 0) ? 1u : 0u);
                         umma_commit(bar_empty + 8 * s);      // frees the stage when these MMAs have read it
-                        fill++;
+                        if (++s == S) { s = 0; ph ^= 1; }
                     }
                     if (ok) umma_commit(bar_accf + 8 * buf);  // accumulator of this piece complete
                 }
