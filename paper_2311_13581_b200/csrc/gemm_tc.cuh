@@ -115,6 +115,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: false when the CTA is giving up (another role timed out, or this wait did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* g_status) {
+    if (mbar_try_wait(bar, parity)) return true;          // the usual case costs no clock read
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
