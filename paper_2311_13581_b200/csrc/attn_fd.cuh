@@ -229,8 +229,25 @@ k_attn_fd(const AttnParams p) {
     }
     cp_async_commit();
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Three trips to L2 start here and overlap: the row tables (final now), the queries, and - once the tables are
+    // in - the blocks that were not fetched early.  The queries are asked for before anything waits for the tables.
+    const int seq_f = __ldcg(p.row_seq + row0), len_f = __ldcg(p.row_pos + row0);    // the same for every thread
+    float2 qraw[DH / 16][4];
     {
-        const int seq_f = __ldcg(p.row_seq + row0), len_f = __ldcg(p.row_pos + row0);    // final now, the same for every thread
+        const int i0 = mt * 16 + g, i1 = i0 + 8;
+        const float* q0 = p.q + (size_t)(row0 + i0) * p.ldq + head * DH;
+        const float* q1 = p.q + (size_t)(row0 + i1) * p.ldq + head * DH;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ks++) {
+            const int c = ks * 16 + 2 * t;
+            const float2 z = make_float2(0.f, 0.f);
+            qraw[ks][0] = i0 < M ? *reinterpret_cast<const float2*>(q0 + c) : z;
+            qraw[ks][1] = i1 < M ? *reinterpret_cast<const float2*>(q1 + c) : z;
+            qraw[ks][2] = i0 < M ? *reinterpret_cast<const float2*>(q0 + c + 8) : z;
+            qraw[ks][3] = i1 < M ? *reinterpret_cast<const float2*>(q1 + c + 8) : z;
+        }
+    }
+    {
         if (seq_f != seq || len_f != len) {
             // the early part worked from tables of an earlier step: let its copies land, then start over
             cp_async_wait<0>();
@@ -251,19 +268,11 @@ k_attn_fd(const AttnParams p) {
     uint32_t qf[DH / 16][4], qfl[DH / 16][4];
     {
         const float sc = 1.4426950408889634f * rsqrtf((float)DH);
-        const int i0 = mt * 16 + g, i1 = i0 + 8;
-        const float* q0 = p.q + (size_t)(row0 + i0) * p.ldq + head * DH;
-        const float* q1 = p.q + (size_t)(row0 + i1) * p.ldq + head * DH;
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ks++) {
-            const int c = ks * 16 + 2 * t;
-            float2 a = make_float2(0.f, 0.f), bq = a, c2 = a, d2 = a;
-            if (i0 < M) { a = *reinterpret_cast<const float2*>(q0 + c); c2 = *reinterpret_cast<const float2*>(q0 + c + 8); }
-            if (i1 < M) { bq = *reinterpret_cast<const float2*>(q1 + c); d2 = *reinterpret_cast<const float2*>(q1 + c + 8); }
-            const float2 f4[4] = {a, bq, c2, d2};
 #pragma unroll
             for (int e = 0; e < 4; e++) {
-                const float x = f4[e].x * sc, y = f4[e].y * sc;
+                const float x = qraw[ks][e].x * sc, y = qraw[ks][e].y * sc;
                 const __nv_bfloat162 hi = __floats2bfloat162_rn(x, y);
                 qf[ks][e] = *reinterpret_cast<const uint32_t*>(&hi);
                 qfl[ks][e] = pack_bf16(x - __low2float(hi), y - __high2float(hi));
