@@ -520,6 +520,9 @@ __device__ __forceinline__ void ll_reset(float* first, size_t stride, int n_othe
 // so a launch ends without any bookkeeping.  All CTAs of the grid are resident (one per SM), the counter
 // only ever waits for work of an EARLIER GEMM, and every wait is bounded.
 constexpr int kMaxOps = 4;
+// pieces of a CTA per GEMM that are worked out once and kept in shared memory.  A CTA has at most
+// n_tiles / CTAs + 2 pieces (whole tiles plus at most two streamed ones)
+constexpr int kPieceCache = 16;
 struct ChainMaps { CUtensorMap m[kMaxOps][4]; };      // per GEMM: weight maps 0..2, activation map
 struct ChainParams {
     int n_ops;
@@ -605,7 +608,6 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
     __shared__ float s_x[(MANY ? kEpiGroups : 1) * 128 * 9];
     // this CTA's pieces of every GEMM of the chain, worked out once (the schedule arithmetic uses
     // 64-bit divisions, which would otherwise sit between two pieces on every role's critical path)
-    constexpr int kPieceCache = 16;
     __shared__ Piece s_piece[kMaxOps][kPieceCache];
     __shared__ int s_piece_ok[kMaxOps][kPieceCache];
 
@@ -626,7 +628,10 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
             out = s_piece[oi][it];
             return true;
         }
-        return get_piece(cp.op[oi], cta, G, it, out);
+        // (the step's kernels never get here: the host sends a launch whose CTAs have more pieces than the cache
+        // holds to the traced instantiation, which like the prompt-chunk one keeps the arithmetic)
+        if (BIG || TRACE) return get_piece(cp.op[oi], cta, G, it, out);
+        return false;
     };
     const uint32_t stage_bytes = kATileBytes + cp.npad * 128;
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;

@@ -446,7 +446,9 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     const size_t smem = (size_t)cp.stages * (kATileBytes + cp.npad * 128) + 1024;
     const bool big = ops[0].p.whole_only != 0;        // a prompt chunk: the kernel instance with token tiles
     const bool many = !big && ops[0].p.R >= kManyRowsFrom;        // the instance with several epilogue groups
-    const bool dbg = c->trace || cp.test_stuck || cp.hold;      // stamps, test hook, held-back requests: the instance that has them
+    bool dbg = c->trace || cp.test_stuck || cp.hold;      // stamps, test hook, held-back requests: the instance that has them
+    // ... and the schedule arithmetic for CTAs with more pieces than the kernel keeps in shared memory
+    for (int j = 0; j < n_ops; j++) dbg |= ops[j].p.n_tiles / c->n_sms + 2 > kPieceCache;
     auto kern = big ? k_gemm_tc_big : many ? k_gemm_tc_many : dbg ? k_gemm_tc_traced : k_gemm_tc;
     size_t& smem_set = big ? c->gemm_big_smem_set : many ? c->gemm_many_smem_set : dbg ? c->gemm_traced_smem_set : c->gemm_smem_set;
     if (smem > smem_set) {
