@@ -291,9 +291,10 @@ int pass_set_state(pass_ctx *ctx, int seq, int len, int32_t pending);
 #define PASS_DBG_TRACE         9  /* uint64 [launch][4 GEMMs][CTAs][8]: %globaltimer stamps of the GEMM-chain
                                      launches since the last read, when PASS_TRACE is set in the environment:
                                      activations available, first tile ready, last MMA issued, epilogues done */
-#define PASS_DBG_FOOTPRINT    10  /* int32 [6]: shared memory in bytes of the step's GEMM kernel (static, dynamic at 9..16
-                                     rows) and of its attention kernel (static, dynamic), the SM's total and what the
-                                     system reserves per block: the two kernels are meant to fit on one SM together */
+#define PASS_DBG_FOOTPRINT    10  /* int32 [6] or [9]: shared memory in bytes of the step's GEMM kernel (static, dynamic at up
+                                     to 9 rows) and of its attention kernel (static, dynamic), the SM's total and what the
+                                     system reserves per block; with room for 9 values also the registers of a CTA of
+                                     each and the SM's register file: the two kernels are meant to fit on one SM together */
 #define PASS_DBG_ATTN_TRACE   11  /* uint64 [launch][16][16][8]: stamps of the long-cache attention kernel's launches since
                                      the last read (PASS_TRACE set, one sequence): per (head / 4, key slice) of every
                                      fourth head: entry, dependency wait over, first key block in shared memory, last

@@ -263,7 +263,7 @@ class PassContext:
         elif what == PASS_DBG_STATUS:
             a = np.empty(1, dtype=np.int32)
         elif what == PASS_DBG_FOOTPRINT:
-            a = np.empty(6, dtype=np.int32)
+            a = np.empty(9, dtype=np.int32)
         else:
             a = np.empty(B, dtype=np.int32)
         _check(self.lib, self.lib.pass_get_debug(self.h, what, a.ctypes.data, a.nbytes))

@@ -1366,6 +1366,14 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         o[3] = 2 * kAttnStages * kAttnBK * c->md.dh * 2;
         o[4] = sm_total;
         o[5] = reserved;
+        if (bytes >= 9 * 4) {
+            // registers: allocated in units of 8 per thread; the two CTAs must fit the SM's register file together
+            int regs_total = 0;
+            CUDA_TRY(cudaDeviceGetAttribute(&regs_total, cudaDevAttrMaxRegistersPerMultiprocessor, dev));
+            o[6] = ((ag.numRegs + 7) / 8) * 8 * kGemmThreads;
+            o[7] = ((aa.numRegs + 7) / 8) * 8 * 128;
+            o[8] = regs_total;
+        }
         return PASS_OK;
     }
     if (what == PASS_DBG_STATUS) {

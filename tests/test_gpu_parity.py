@@ -35,12 +35,15 @@ def test_library_loaded_and_device_is_blackwell():
 def test_gemm_and_attention_ctas_fit_on_one_sm_together():
     """The attention kernel's CTA and the CTA of the GEMM launch after it are meant to be resident side by
     side (the GEMM launch streams weights while attention runs: 0.12 ms of a 3.06 ms step at the 7B shape).
-    Their shared memory fills an SM to within a few hundred bytes, so the sum is checked here."""
+    Their shared memory fills an SM to within a few hundred bytes and their registers its register file to within
+    a thousand, so both sums are checked here."""
     pb = _pb()
     shape = dataclasses.replace(TINY_BF16, d_head=128, n_heads=2)       # heads of 128, as in the 7B and 13B shapes
     ctx = pb.PassContext(shape, si.weights_to(si.make_weights(shape, seed=1), "cuda:0"), 1, 64)
-    g_static, g_dyn, a_static, a_dyn, sm_total, reserved = [int(x) for x in ctx.get_debug(pb.PASS_DBG_FOOTPRINT)]
-    assert g_static + g_dyn + reserved + a_static + a_dyn + reserved <= sm_total, (g_static, g_dyn, a_static, a_dyn, sm_total, reserved)
+    fp = [int(x) for x in ctx.get_debug(pb.PASS_DBG_FOOTPRINT)]
+    g_static, g_dyn, a_static, a_dyn, sm_total, reserved, g_regs, a_regs, regs_total = fp
+    assert g_static + g_dyn + reserved + a_static + a_dyn + reserved <= sm_total, fp
+    assert 0 < g_regs and 0 < a_regs and g_regs + a_regs <= regs_total, fp
     ctx.close()
 
 
