@@ -377,7 +377,7 @@ int pass_linear_noalloc(pass_ctx *ctx, int which, int layer, const float *x_devi
  *       positions shorter than it is, which forces its re-check and restart path.
  *   PASS_HOOK_ATTN_LONG_FROM, value n >= 0: a step counts as "long" (other attention launch shape; with
  *       d_head 128 and at most 16 rows per sequence the tcgen05 attention kernel) as soon as one sequence
- *       has n cached positions.  Default 3072 (PASS_ATTN_LONG_FROM in the environment at creation); 0
+ *       has n cached positions.  Default 3584 (PASS_ATTN_LONG_FROM in the environment at creation); 0
  *       sends every step down the long path, so that small test cases reach it.
  *   PASS_HOOK_ATTN_STUCK, value 0/1: the tcgen05 attention kernel never announces its scores, so its
  *       bounded waits run out; the call returns PASS_ERR_TIMEOUT with the sequence state untouched.

@@ -153,7 +153,7 @@ struct pass_ctx {
     int n_sms = 148;
     bool use_pdl = true;
     bool attn_long = false;       // this step's contexts are long: twice as many attention slices (see step_launch)
-    int attn_long_from = 3072;    // PASS_ATTN_LONG_FROM: cached positions from which a step counts as long
+    int attn_long_from = 3584;    // PASS_ATTN_LONG_FROM: cached positions from which a step counts as long
     bool attn_tc = true;          // PASS_ATTN_NO_TC: long contexts keep the mma.sync kernel (k_attn_tc otherwise, d_head 128, <= 16 rows)
     bool attn_tc_ready = false, attn_tc_smem_set = false;
     AttnTcMaps attn_tc_maps;      // the key and the value cache as matrices of 128 columns
