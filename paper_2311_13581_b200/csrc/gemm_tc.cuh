@@ -1136,7 +1136,11 @@ k_gemm_tc_traced(const __grid_constant__ ChainMaps maps, const __grid_constant__
 constexpr int kGemmThreadsMany = 128 + kEpiGroups * 128;
 __global__ void __launch_bounds__(kGemmThreadsMany, 1)
 k_gemm_tc_many(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
-    gemm_chain_body<false, true>(maps, cp);
+    gemm_chain_body<false, true, false>(maps, cp);
+}
+__global__ void __launch_bounds__(kGemmThreadsMany, 1)
+k_gemm_tc_many_traced(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    gemm_chain_body<false, true, true>(maps, cp);
 }
 // prompt chunks: alone on its SM (192 KB of ring), so the register cap of the step's kernel does not apply
 __global__ void __launch_bounds__(kGemmThreads, 1)

@@ -163,7 +163,7 @@ struct pass_ctx {
     int gemm_test_stuck = 0;      // pass_debug_set(PASS_HOOK_GEMM_STUCK, 1): contributors withhold their partial sums
     // Function attributes and occupancy answers belong to the device the context lives on, so they are
     // remembered per context, never per process.
-    size_t gemm_smem_set = 0, gemm_big_smem_set = 0, gemm_many_smem_set = 0, gemm_traced_smem_set = 0;
+    size_t gemm_smem_set = 0, gemm_big_smem_set = 0, gemm_many_smem_set = 0, gemm_traced_smem_set = 0, gemm_many_traced_smem_set = 0;
     std::map<int, bool> attn_attr_set;         // by kernel instance
     std::map<int, int> attn_cluster_max;       // by kernel instance, slice count and sequences
     cudaError_t launch_err = cudaSuccess;      // first failed launch / attribute call since the last check
@@ -449,8 +449,8 @@ static void launch_chain(pass_ctx* c, ChainOp* ops, int n_ops) {
     bool dbg = c->trace || cp.test_stuck || cp.hold;      // stamps, test hook, held-back requests: the instance that has them
     // ... and the schedule arithmetic for CTAs with more pieces than the kernel keeps in shared memory
     for (int j = 0; j < n_ops; j++) dbg |= ops[j].p.n_tiles / c->n_sms + 2 > kPieceCache;
-    auto kern = big ? k_gemm_tc_big : many ? k_gemm_tc_many : dbg ? k_gemm_tc_traced : k_gemm_tc;
-    size_t& smem_set = big ? c->gemm_big_smem_set : many ? c->gemm_many_smem_set : dbg ? c->gemm_traced_smem_set : c->gemm_smem_set;
+    auto kern = big ? k_gemm_tc_big : many ? (dbg ? k_gemm_tc_many_traced : k_gemm_tc_many) : dbg ? k_gemm_tc_traced : k_gemm_tc;
+    size_t& smem_set = big ? c->gemm_big_smem_set : many ? (dbg ? c->gemm_many_traced_smem_set : c->gemm_many_smem_set) : dbg ? c->gemm_traced_smem_set : c->gemm_smem_set;
     if (smem > smem_set) {
         note_err(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "k_gemm_tc shared memory size");
         // all of the SM's L1/shared storage as shared memory: lets the CTA of the next launch become
