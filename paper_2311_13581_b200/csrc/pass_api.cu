@@ -146,7 +146,7 @@ struct pass_ctx {
     // tensor-core path (bf16 models)
     __nv_bfloat16 *d_xn_bf = nullptr, *d_attn_bf = nullptr, *d_act_bf = nullptr;
     float *d_q_out = nullptr, *d_sumsq_a = nullptr, *d_sumsq_b = nullptr, *d_partial = nullptr;
-    float* d_ll = nullptr;             // hand-over slots of the <=16-row GEMMs, all bits set when idle
+    float* d_ll = nullptr;             // hand-over slots of the step's GEMMs (EMPTY-or-value words), all bits set when idle
     int* d_counters = nullptr;
     float *d_attn_po = nullptr, *d_attn_pml = nullptr;
     int* d_attn_cnt = nullptr;
@@ -946,7 +946,7 @@ int pass_create(const pass_config* cfg, void* kv_k, void* kv_v, size_t kv_bytes,
     if (cudaMemsetAsync(w, 0, L.h, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.xn_bf, 0, L.packed - L.xn_bf, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
-    // the hand-over slots of the <=16-row GEMMs are EMPTY (all bits set) whenever no launch is using them
+    // the hand-over slots of the step's GEMMs are EMPTY (all bits set) whenever no launch is using them
     if (cfg->dtype == PASS_DTYPE_BF16 &&
         cudaMemsetAsync(w + L.ll_ws, 0xFF, kLLRegionBytes * kMaxOps, c->stream) != cudaSuccess) return fail(PASS_ERR_CUDA);
     // stamps are told from empty slots by being non-zero

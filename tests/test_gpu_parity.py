@@ -34,7 +34,7 @@ def test_library_loaded_and_device_is_blackwell():
 
 def test_gemm_and_attention_ctas_fit_on_one_sm_together():
     """The attention kernel's CTA and the CTA of the GEMM launch after it are meant to be resident side by
-    side (the GEMM launch streams weights while attention runs: 0.12 ms of a 3.06 ms step at the 7B shape).
+    side (the GEMM launch streams weights while attention runs: 0.12 ms of a step at the 7B shape).
     Their shared memory fills an SM to within a few hundred bytes and their registers its register file to within
     a thousand, so both sums are checked here."""
     pb = _pb()
