@@ -137,6 +137,11 @@ class PassContext:
         self.device = torch.device(device)
         self.B = int(max_batch)
         self.k_max = int(shape.k_max)
+        # result buffers of step / step_collect, made once: building arrays and their ctypes views per call costs
+        # the caller some 15 us of a 2.8 ms step
+        self._out = np.full((self.B, self.k_max + 1), -1, dtype=np.int32)
+        self._n = np.zeros(self.B, dtype=np.int32)
+        self._out_ptr, self._n_ptr = self._out.ctypes.data, self._n.ctypes.data
         self.vocab = int(shape.vocab)
         cfg = _Config(shape.n_layers, shape.d_model, shape.n_heads, shape.d_head, shape.d_ffn, shape.vocab,
                       shape.k_max, self.B, int(kv_capacity), 0 if shape.dtype == "fp32" else 1,
@@ -181,24 +186,22 @@ class PassContext:
     def step(self, k: int, temperature: float, uniforms: Optional[np.ndarray]
              ) -> Tuple[List[List[int]], np.ndarray]:
         """uniforms: [B][2k+1] float32 host array (None iff temperature == 0)."""
-        out = np.full((self.B, self.k_max + 1), -1, dtype=np.int32)
-        n = np.zeros(self.B, dtype=np.int32)
+        out, n = self._out, self._n
         up = None
         if uniforms is not None:
             u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(self.B, 2 * k + 1)
             up = u.ctypes.data
-        _check(self.lib, self.lib.pass_step(self.h, k, float(temperature), up, out.ctypes.data, n.ctypes.data))
-        return [out[b, :n[b]].tolist() for b in range(self.B)], n
+        _check(self.lib, self.lib.pass_step(self.h, k, float(temperature), up, self._out_ptr, self._n_ptr))
+        return [out[b, :n[b]].tolist() for b in range(self.B)], n.copy()
 
     def step_enqueue(self, k: int, temperature: float, uniforms_device=None) -> None:
         p = None if uniforms_device is None else uniforms_device.data_ptr()
         _check(self.lib, self.lib.pass_step_enqueue(self.h, k, float(temperature), p))
 
     def step_collect(self) -> Tuple[List[List[int]], np.ndarray]:
-        out = np.full((self.B, self.k_max + 1), -1, dtype=np.int32)
-        n = np.zeros(self.B, dtype=np.int32)
-        _check(self.lib, self.lib.pass_step_collect(self.h, out.ctypes.data, n.ctypes.data))
-        return [out[b, :n[b]].tolist() for b in range(self.B)], n
+        out, n = self._out, self._n
+        _check(self.lib, self.lib.pass_step_collect(self.h, self._out_ptr, self._n_ptr))
+        return [out[b, :n[b]].tolist() for b in range(self.B)], n.copy()
 
     def forward_tokens(self, seq: int, tokens: Sequence[int], commit: int, want_logits: bool = True):
         a = np.ascontiguousarray(tokens, dtype=np.int32)
