@@ -147,18 +147,20 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
     return v;
 }
 
-// Registers: a decode-step CTA (ring of three stages) shares its SM with the step's GEMM CTA, which takes 136
+// Registers (NREG): the CTA of a step of up to nine rows shares its SM with the step's GEMM CTA, which takes 136
 // registers x 256 threads, so 232 x 128 are left for it - and it is measurably faster with them than with 168
-// (2.796 -> 2.778 ms per step at 512 cached positions, 3.077 -> 3.005 ms at 2048).  With a ring of two stages
-// three of these CTAs share an SM: 168.
+// (2.796 -> 2.778 ms per step at 512 cached positions, 3.077 -> 3.005 ms at 2048).  Where three of these CTAs
+// share an SM (steps of ten rows or more): 168.
 // MT = m-tiles of 16 rows per CTA (4 warps: MT = 4 gives every warp its own 16 rows and all keys of a block,
 // the usual flash-attention split for many rows).  HL = queries and probabilities as bf16 hi + lo pairs;
 // without it they are single bf16 values (prompt chunks in plain bf16, half the MMAs).
 // CHUNK = the rows are one sequence's prompt chunk (rows_per_block, out_tile_rows, optional lo parts); the
-// decode step's instances have it off and carry none of that code.  ST = depth of the key / value ring: 3 where the
-// CTA shares its SM with the next GEMM launch's CTA, 2 (64 KB at d_head 128) where three of these CTAs share an SM.
-template <int DH, int MT, bool CL, bool HL = true, bool CHUNK = false, int ST = kAttnStages>
-__global__ void __maxnreg__(ST == 2 ? 168 : 232)
+// decode step's instances have it off and carry none of that code.  ST = depth of the key / value ring: 2 (64 KB at
+// d_head 128) in the decode step - beside the GEMM CTA a third stage buys nothing, a seventh stage of the GEMM's
+// ring does (2.778 -> 2.748 ms), and three CTAs of two stages fit an SM where they have it to themselves -, 3
+// for prompt chunks and the doubled slices of long caches.
+template <int DH, int MT, bool CL, bool HL = true, bool CHUNK = false, int ST = kAttnStages, int NREG = 232>
+__global__ void __maxnreg__(NREG)
 k_attn_fd(const AttnParams p) {
     extern __shared__ __align__(128) uint8_t smem_attn[];
     constexpr int CH = DH / 8;                       // 16-byte chunks per key

@@ -601,8 +601,8 @@ __device__ __forceinline__ void gemm_chain_body(const ChainMaps& maps, const Cha
     __shared__ int s_epi_done;
     __shared__ int s_last;
     __shared__ int s_epi_fail;
-    // (the step's kernel shares its SM with an attention CTA of 96 KB: every byte of static shared memory counts,
-    // 512 bytes more and the two no longer fit side by side)
+    // (the step's kernel shares its SM with an attention CTA of 64 KB and fills the rest with a seventh stage of its
+    // ring: static shared memory that grows by more than 12 KB ends that)
     __shared__ float s_rstd[BIG ? kTokTile : kMaxRows];
     __shared__ unsigned long long s_kvoff[BIG ? kTokTile : kMaxRows];
     __shared__ float s_x[(MANY ? kEpiGroups : 1) * 128 * 9];

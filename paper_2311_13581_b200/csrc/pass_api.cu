@@ -349,7 +349,9 @@ static int gemm_stages(int npad) {
         const int s = atoi(e);
         if (s >= 2 && s <= 16 && (size_t)s * stage + 1024 <= 225 * 1024) return s;
     }
-    int s = (122 * 1024 - 1024) / stage;   // leaves room for one attention CTA (96 KB) beside it
+    // up to 16 padded rows per half: the step's kernel, which leaves room for one attention CTA (ring of two stages:
+    // 64 KB) beside it; more: kernels that have the SM to themselves
+    int s = ((npad > 32 ? 200 : 142) * 1024 - 1024) / stage;
     if (s < 4) s = std::min(4, (220 * 1024) / stage);
     return std::max(2, std::min(16, s));
 }
@@ -492,13 +494,13 @@ static void launch_gemm(pass_ctx* c, const CUtensorMap& a0, const CUtensorMap& a
 
 // The bf16 decoder layers on tensor cores.  Per layer: QKV GEMM (+RMSNorm factor, rotary, KV append),
 // attention, O GEMM (+residual, next norm's input), gate/up GEMM (+SwiGLU), down GEMM (+residual).
-template <int DH, int MT, bool CL, int ST>
+template <int DH, int MT, bool CL, int ST, int NREG>
 static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     constexpr int smem = 2 * ST * kAttnBK * DH * 2;
-    bool& set = c->attn_attr_set[ST * 4096 + DH * 8 + MT * 2 + (CL ? 1 : 0)];
+    bool& set = c->attn_attr_set[NREG * 65536 + ST * 4096 + DH * 8 + MT * 2 + (CL ? 1 : 0)];
     if (!set) {
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST>, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_attn_fd carveout");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST, NREG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, CL, true, false, ST, NREG>, cudaFuncAttributePreferredSharedMemoryCarveout, 100), "k_attn_fd carveout");
         set = true;
     }
     cudaLaunchConfig_t cfg;
@@ -521,7 +523,7 @@ static void launch_attn_fd_impl(pass_ctx* c, const AttnParams& ap, int n_seq) {
     }
     cfg.attrs = at;
     cfg.numAttrs = na;
-    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL, true, false, ST>, ap), "k_attn_fd launch");
+    note_err(c, cudaLaunchKernelEx(&cfg, k_attn_fd<DH, MT, CL, true, false, ST, NREG>, ap), "k_attn_fd launch");
     c->launches++;
 }
 
@@ -553,14 +555,14 @@ static void launch_attn_tc(pass_ctx* c, const AttnParams& ap_in, int n_seq) {
 // Can the slices of every (sequence, head) run as one cluster each, all at the same time?  Asked once per
 // context, kernel instance, slice count and batch; if not (or with more than 8 slices) the merge goes through
 // global memory.
-template <int DH, int MT, int ST>
+template <int DH, int MT, int ST, int NREG>
 static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
     if (!c->attn_cluster || n_split < 2 || n_split > 8) return false;
-    const int key = (((ST * 256 + DH) * 8 + MT) * 32 + n_split) * 256 + n_seq;
+    const int key = ((((NREG / 64) * 4 + ST) * 256 + DH) * 8 + MT) * 32 * 256 + n_split * 256 + n_seq;
     auto it = c->attn_cluster_max.find(key);
     if (it == c->attn_cluster_max.end()) {
         constexpr int smem = 2 * ST * kAttnBK * DH * 2;
-        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, true, true, false, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
+        note_err(c, cudaFuncSetAttribute(k_attn_fd<DH, MT, true, true, false, ST, NREG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem), "k_attn_fd shared memory size");
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
         cfg.gridDim = dim3(c->md.H, n_seq, n_split);
@@ -572,16 +574,16 @@ static bool attn_cluster_ok(pass_ctx* c, int n_split, int n_seq) {
         cfg.attrs = at;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true, true, false, ST>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
+        if (cudaOccupancyMaxActiveClusters(&n, k_attn_fd<DH, MT, true, true, false, ST, NREG>, &cfg) != cudaSuccess) { n = 0; cudaGetLastError(); }
         it = c->attn_cluster_max.emplace(key, n).first;
     }
     return it->second >= c->md.H * n_seq;
 }
 
-template <int DH, int MT, int ST = kAttnStages>
+template <int DH, int MT, int ST, int NREG>
 static void launch_attn_fd(pass_ctx* c, const AttnParams& ap, int n_seq) {
-    if (attn_cluster_ok<DH, MT, ST>(c, ap.n_split, n_seq)) launch_attn_fd_impl<DH, MT, true, ST>(c, ap, n_seq);
-    else launch_attn_fd_impl<DH, MT, false, ST>(c, ap, n_seq);
+    if (attn_cluster_ok<DH, MT, ST, NREG>(c, ap.n_split, n_seq)) launch_attn_fd_impl<DH, MT, true, ST, NREG>(c, ap, n_seq);
+    else launch_attn_fd_impl<DH, MT, false, ST, NREG>(c, ap, n_seq);
 }
 
 // GEMMs of the decoder layers as chain entries.
@@ -727,16 +729,20 @@ static int enqueue_layers_tc(pass_ctx* c, int R, int n_seq, bool head, bool inpu
             const int pairs = md.H * n_seq;
             ap.n_split = std::max(1, std::min(8, 3 * c->n_sms / pairs));
             ap.n_split = std::min(ap.n_split, (2 * kMaxCtas + pairs) / pairs);      // what the slices' workspace holds
-            if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1, 2>(c, ap, n_seq); else launch_attn_fd<128, 2, 2>(c, ap, n_seq); }
-            else              { if (M <= 16) launch_attn_fd<64, 1, 2>(c, ap, n_seq); else launch_attn_fd<64, 2, 2>(c, ap, n_seq); }
+            if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1, 2, 168>(c, ap, n_seq); else launch_attn_fd<128, 2, 2, 168>(c, ap, n_seq); }
+            else              { if (M <= 16) launch_attn_fd<64, 1, 2, 168>(c, ap, n_seq); else launch_attn_fd<64, 2, 2, 168>(c, ap, n_seq); }
         } else if (M <= 32) {
             // at most one CTA per SM: the next GEMM's CTA then fits beside it and prefetches weights
             ap.n_split = std::max(1, std::min(kAttnMaxSplit, c->n_sms / (md.H * n_seq)));
             // Long contexts: the key loop (tensor-core work of 4 warps) outweighs everything that one CTA per
             // SM buys at short contexts, so the slices are doubled - two CTAs per SM, 8 warps on the keys.
-            if (c->attn_long && ap.n_split * 2 <= 8) ap.n_split *= 2;
-            if (md.dh == 128) { if (M <= 16) launch_attn_fd<128, 1>(c, ap, n_seq); else launch_attn_fd<128, 2>(c, ap, n_seq); }
-            else              { if (M <= 16) launch_attn_fd<64, 1>(c, ap, n_seq); else launch_attn_fd<64, 2>(c, ap, n_seq); }
+            // (at most nine rows here: one 16-row tile)
+            if (c->attn_long && ap.n_split * 2 <= 8) {
+                ap.n_split *= 2;
+                if (md.dh == 128) launch_attn_fd<128, 1, 3, 232>(c, ap, n_seq); else launch_attn_fd<64, 1, 3, 232>(c, ap, n_seq);
+            } else {
+                if (md.dh == 128) launch_attn_fd<128, 1, 2, 232>(c, ap, n_seq); else launch_attn_fd<64, 1, 2, 232>(c, ap, n_seq);
+            }
         } else {
             // more than 32 rows: one sequence's prompt chunk (pass_forward_tokens, pass_prefill)
             ap.debug_stale = 0;
@@ -1353,8 +1359,8 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         if (!c->use_tc) return PASS_ERR_STATE;
         cudaFuncAttributes ag, aa;
         CUDA_TRY(cudaFuncGetAttributes(&ag, k_gemm_tc));
-        if (c->md.dh == 128) CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<128, 1, true>));
-        else CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<64, 1, true>));
+        if (c->md.dh == 128) CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<128, 1, true, true, false, 2, 232>));
+        else CUDA_TRY(cudaFuncGetAttributes(&aa, k_attn_fd<64, 1, true, true, false, 2, 232>));
         int dev = 0, sm_total = 0, reserved = 0;
         CUDA_TRY(cudaGetDevice(&dev));
         CUDA_TRY(cudaDeviceGetAttribute(&sm_total, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
@@ -1363,7 +1369,7 @@ int pass_get_debug(pass_ctx* c, int what, void* dst, size_t bytes) {
         o[0] = (int)ag.sharedSizeBytes;
         o[1] = gemm_stages(32) * (kATileBytes + 32 * 128) + 1024;
         o[2] = (int)aa.sharedSizeBytes;
-        o[3] = 2 * kAttnStages * kAttnBK * c->md.dh * 2;
+        o[3] = 2 * 2 * kAttnBK * c->md.dh * 2;          // ring of two stages
         o[4] = sm_total;
         o[5] = reserved;
         if (bytes >= 9 * 4) {
