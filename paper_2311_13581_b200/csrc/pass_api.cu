@@ -351,7 +351,8 @@ static int gemm_stages(int npad) {
     }
     // up to 16 padded rows per half: the step's kernel, which leaves room for one attention CTA (ring of two stages:
     // 64 KB) beside it; more: kernels that have the SM to themselves
-    int s = ((npad > 32 ? 200 : 142) * 1024 - 1024) / stage;
+    // (measured: more than eight stages make the hand-overs slower again - k = 8: 3.460 / 3.480 ms with 8 / 9)
+    int s = npad > 32 ? std::min(8, (206 * 1024 - 1024) / stage) : (142 * 1024 - 1024) / stage;
     if (s < 4) s = std::min(4, (220 * 1024) / stage);
     return std::max(2, std::min(16, s));
 }
