@@ -4,7 +4,7 @@
 // head's keys/values exactly once and serves all M <= 32 rows of the sequence from it.
 //
 //   grid  = (heads, sequences, n_split); 128 threads = 4 warps
-//   K/V   : cp.async, 64-key blocks, 3-stage ring in shared memory, 16-byte chunks XOR-swizzled
+//   K/V   : cp.async, 64-key blocks, a ring of two or three stages in shared memory, 16-byte chunks XOR-swizzled
 //   math  : mma.sync m16n8k16 bf16 (S = Q K^T, O += P V), fp32 online softmax per warp
 //   split : each slice leaves (O, max, sum) partials; the last slice to finish (counter per
 //           sequence and head) merges them in slice order and writes the bf16 hi/lo rows that
